@@ -1,0 +1,149 @@
+/*
+ * plogp.h — C ABI of the pLogP collective-communication tuner for one NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates, on the GPU, the completion-time models that "Fast Tuning of
+ * Intra-Cluster Collective Communications" (Barchet-Estefanel & Mounié) prints for the
+ * Broadcast strategies (Table 1) and the Scatter strategies (Table 2), searches the segment
+ * size that minimises each segmented model (Section 3.1) and selects, for every parameter set
+ * (communication pattern, message size, number of processes — Section 1), the strategy with the
+ * lowest predicted time (Sections 1 and 5).  The network enters through the pLogP parameters
+ * of Section 2: the latency L and the gap g(m), measured at a list of message sizes.
+ *
+ * All arithmetic is IEEE double.  There is no CPU fallback: every call needs a CUDA device of
+ * compute capability 10.0.
+ *
+ * Strategy ids (Table 1 rows in print order, then Table 2 rows):
+ *    0 Flat Tree                  (P-1) g(m) + L
+ *    1 Flat Tree Rendezvous       (P-1) g(m) + 2 g(1) + 3 L
+ *    2 Segmented Flat Tree        (P-1) (g(s) k) + L
+ *    3 Chain                      (P-1) (g(m) + L)
+ *    4 Chain Rendezvous           (P-1) (g(m) + 2 g(1) + 3 L)
+ *    5 Segmented Chain (Pipeline) (P-1) (g(s) + L) + g(s) (k-1)
+ *    6 Binary Tree                ceil(log2 P) (2 g(m) + L)      (printed as an upper bound)
+ *    7 Binomial Tree              floor(log2 P) g(m) + ceil(log2 P) L
+ *    8 Binomial Tree Rendezvous   floor(log2 P) g(m) + ceil(log2 P) (2 g(1) + 3 L)
+ *    9 Segmented Binomial Tree    floor(log2 P) g(s) k + ceil(log2 P) L
+ *   10 Scatter Flat Tree          (P-1) g(m) + L
+ *   11 Scatter Chain              sum_{j=1..P-1} g(j m) + (P-1) L
+ *   12 Scatter Binomial Tree      sum_{j=0..ceil(log2 P)-1} g(2^j m) + ceil(log2 P) L
+ *
+ * Conventions the paper leaves open (fixed here, identical in every entry point):
+ *   - g(x) is linear in x (bytes) between neighbouring measured sizes; below the first size it
+ *     keeps the first value; above the last size the last interval's line is continued.
+ *   - k, the number of segments of Section 2, is ceil(m/s) (k_mode 0) or floor(m/s) as Section
+ *     3.1 prints it (k_mode 1); every segment costs g(s).
+ *   - candidate segment sizes for a message m are the grid values s <= m; if none fits, the
+ *     message is sent whole (s = m, k = 1) and best_s reports m.
+ *   - ties: the smallest segment size, then the lowest strategy id.
+ *
+ * Threading: calls on one plogp_tables handle must not overlap in time on the host, and their
+ * device work must be ordered (use one stream, or order the streams yourself): a handle owns
+ * device scratch that its calls reuse.  Different handles are independent.
+ */
+#ifndef PLOGP_H
+#define PLOGP_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PLOGP_N_STRATEGIES 13
+#define PLOGP_N_SEGMENTED 3      /* ids 2, 5, 9, in this order in best_s outputs */
+#define PLOGP_MAX_BREAKPOINTS 1024
+#define PLOGP_MAX_INLINE_S 64    /* informational: longer segment lists go through the sweep kernel */
+
+typedef enum {
+    PLOGP_OK = 0,
+    PLOGP_E_INVAL = -1, /* malformed argument (null pointer, n_bp < 2, sizes not increasing, NaN or negative
+                           gap, P < 2, m or s not a positive multiple of dtype_bytes, lists not ascending) */
+    PLOGP_E_NOMEM = -2, /* host or device allocation failed */
+    PLOGP_E_CUDA = -3,  /* a CUDA runtime call failed; plogp_last_cuda_error() names it */
+    PLOGP_E_RANGE = -4  /* m, s or a table size too large: m and s must be < 2^32, sizes < 2^53,
+                           n_bp <= PLOGP_MAX_BREAKPOINTS, (P_hi - 1) * m < 2^53 */
+} plogp_status;
+
+/* Opaque set of pLogP parameter tables resident on the current CUDA device. */
+typedef struct plogp_tables plogp_tables;
+
+/*
+ * Upload n_tables independent pLogP parameter sets (Section 2: gap g at n_bp message sizes and
+ * the latency L of each network).
+ *   sizes_bytes  HOST, [n_bp] when sizes_shared != 0, else [n_tables][n_bp]; strictly increasing.
+ *   gap          HOST, [n_tables][n_bp]; finite, >= 0; any time unit (the outputs use the same).
+ *   latency      HOST, [n_tables]; finite, >= 0.
+ *   out          receives the handle; release it with plogp_table_free.
+ * The host arrays are copied before the call returns; the caller keeps them.  The call
+ * synchronises with the device (it allocates).  Nothing is written to *out on error.
+ */
+int plogp_table_load(int n_tables, int n_bp, const uint64_t *sizes_bytes, int sizes_shared,
+                     const double *gap, const double *latency, plogp_tables **out);
+
+/* Release a handle and its device memory (synchronises). NULL is accepted. */
+int plogp_table_free(plogp_tables *tables);
+
+/*
+ * The parameter sets to evaluate: process counts P, message sizes m (Section 1's "message size,
+ * number of processes") and candidate segment sizes s (Section 2: a multiple of the basic
+ * datatype's size).  All arrays are HOST memory and are copied by the call.
+ */
+typedef struct {
+    const int32_t *P;   /* [n_P] ascending, each >= 2; or NULL for the contiguous range P_lo..P_hi */
+    int32_t n_P;        /* ignored when P == NULL */
+    int32_t P_lo, P_hi; /* used when P == NULL; 2 <= P_lo <= P_hi */
+    const uint64_t *m;  /* [n_m] bytes, ascending, positive multiples of dtype_bytes */
+    int32_t n_m;
+    const uint64_t *s;  /* [n_s] bytes, ascending, positive multiples of dtype_bytes; or NULL for
+                           every s_lo + i * s_step <= s_hi */
+    int64_t n_s;        /* ignored when s == NULL */
+    uint64_t s_lo, s_hi, s_step;
+    uint32_t dtype_bytes;   /* size of the basic datatype, > 0 */
+    uint32_t strategy_mask; /* bit i enables strategy id i */
+    int32_t k_mode;         /* 0: k = ceil(m/s); 1: k = floor(m/s) */
+} plogp_grid;
+
+/*
+ * Evaluate every enabled model of Table 1 / Table 2 on the grid; the segmented ones (ids 2, 5,
+ * 9) are reduced over the candidate segment sizes as Section 3.1 describes.
+ *   d_time    DEVICE, [n_tables][13][n_P][n_m] doubles, m fastest; planes of disabled strategies
+ *             are left untouched.
+ *   d_best_s  DEVICE, [n_tables][3][n_P][n_m] uint32 bytes for ids 2, 5, 9 (disabled: untouched);
+ *             may be NULL.
+ *   stream    a cudaStream_t (NULL = default stream).  Work is enqueued; the call does not wait
+ *             for it, but may synchronise when the handle's scratch has to grow.
+ * Both outputs belong to the caller.
+ */
+int plogp_predict(plogp_tables *tables, const plogp_grid *grid, double *d_time, uint32_t *d_best_s,
+                  void *stream);
+
+/*
+ * Decision table (Sections 1 and 5): for every table, collective (0 = Broadcast, ids 0..9;
+ * 1 = Scatter, ids 10..12), P and m, the enabled strategy with the lowest predicted time.
+ *   d_strategy  DEVICE, uint8  [n_tables][2][n_P][n_m], the winning id
+ *   d_s_bytes   DEVICE, uint32 [n_tables][2][n_P][n_m], its segment size, 0 when unsegmented
+ *   d_time      DEVICE, double [n_tables][2][n_P][n_m], its predicted time
+ * A collective with no enabled strategy leaves its planes untouched.  Same stream and ownership
+ * rules as plogp_predict.
+ */
+int plogp_select_best(plogp_tables *tables, const plogp_grid *grid, uint8_t *d_strategy,
+                      uint32_t *d_s_bytes, double *d_time, void *stream);
+
+/* Static description of a status code. */
+const char *plogp_status_string(int status);
+
+/* Text of the CUDA error behind the calling thread's last PLOGP_E_CUDA ("" if none). */
+const char *plogp_last_cuda_error(void);
+
+/*
+ * Measurement aid with no counterpart in the paper: runs a register-only chain-free stream of
+ * double-precision fused multiply-adds on every SM of the current device for about
+ * `milliseconds` and returns the sustained rate in thread-level FMA instructions per second
+ * (the issue ceiling the segment sweep is compared with).  Synchronises.  Negative on error.
+ */
+double plogp_fp64_fma_rate(double milliseconds);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PLOGP_H */

@@ -1,0 +1,517 @@
+// Host side of the C ABI declared in include/plogp.h: argument validation, table upload, the
+// launch plan for a grid (tiling, chunking of long candidate lists, scratch layout) and the
+// kernel launches.  Every step of the evaluation itself runs in kernels.cu.
+#include "../../include/plogp.h"
+#include "internal.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <limits>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace plogp;
+
+namespace {
+
+thread_local std::string g_cuda_error;
+
+int cuda_fail(cudaError_t e, const char *what)
+{
+    g_cuda_error = std::string(what) + ": " + cudaGetErrorName(e) + " (" + cudaGetErrorString(e) + ")";
+    cudaGetLastError();  // clear the sticky-free error state
+    return PLOGP_E_CUDA;
+}
+
+#define CK(call)                                                  \
+    do {                                                          \
+        cudaError_t e_ = (call);                                  \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call);       \
+    } while (0)
+
+constexpr uint32_t kSegBits = (1u << 2) | (1u << 5) | (1u << 9);
+constexpr uint64_t kTwo32 = 1ull << 32;
+constexpr double kTwo53 = 9007199254740992.0;
+constexpr size_t kSweepScratchLimit = size_t(1) << 30;  // per launch batch of tables
+
+int ceil_log2(int64_t P)
+{
+    int e = 0;
+    while ((int64_t(1) << e) < P) ++e;
+    return e;
+}
+
+// Everything derived from a grid that the launches need; cached on the handle while the same
+// grid keeps being passed.
+struct Plan {
+    std::vector<unsigned char> key;  // serialised grid, for the cache comparison
+    bool empty = true;
+    GridDev G{};
+    int n_seg = 0;
+    bool inline_sweep = true;
+    // fused kernel tiling
+    int n_mtiles = 0, n_ptiles = 1, passes_per_tile = 1;
+    // sweep kernel
+    int n_pairs = 0, sweep_ptiles = 0, chunk_len = 0;
+    size_t off_pair_m = 0, off_pair_chunk = 0, off_pair_row = 0, off_pair_base = 0;
+    int tables_per_batch = 0;
+    size_t scratch_bytes = 0;
+};
+
+}  // namespace
+
+struct plogp_tables {
+    int device = 0;
+    int sm_count = 148;
+    TableDev T{};
+    double *d_tab = nullptr, *d_lat = nullptr;
+    unsigned char *d_grid = nullptr;
+    size_t grid_cap = 0;
+    unsigned char *d_ws = nullptr;
+    size_t ws_cap = 0;
+    Plan plan;
+};
+
+namespace {
+
+template <typename V>
+void put(std::vector<unsigned char> &buf, const V &v)
+{
+    const unsigned char *p = reinterpret_cast<const unsigned char *>(&v);
+    buf.insert(buf.end(), p, p + sizeof(V));
+}
+
+template <typename V>
+void put_array(std::vector<unsigned char> &buf, const V *v, size_t n)
+{
+    const unsigned char *p = reinterpret_cast<const unsigned char *>(v);
+    buf.insert(buf.end(), p, p + n * sizeof(V));
+}
+
+template <typename V>
+size_t append_aligned(std::vector<unsigned char> &blob, const std::vector<V> &v)
+{
+    while (blob.size() % 16) blob.push_back(0);
+    const size_t off = blob.size();
+    put_array(blob, v.data(), v.size());
+    return off;
+}
+
+int validate_grid(const plogp_tables *h, const plogp_grid *g, int64_t *n_s_out)
+{
+    if (!g) return PLOGP_E_INVAL;
+    if (g->strategy_mask >> PLOGP_N_STRATEGIES) return PLOGP_E_INVAL;
+    if (g->k_mode != 0 && g->k_mode != 1) return PLOGP_E_INVAL;
+    if (g->dtype_bytes == 0) return PLOGP_E_INVAL;
+    if (g->n_m < 0) return PLOGP_E_INVAL;
+    if (g->n_m > 0 && !g->m) return PLOGP_E_INVAL;
+    int64_t P_hi;
+    if (g->P) {
+        if (g->n_P < 0) return PLOGP_E_INVAL;
+        for (int i = 0; i < g->n_P; ++i) {
+            if (g->P[i] < 2) return PLOGP_E_INVAL;
+            if (i && g->P[i] <= g->P[i - 1]) return PLOGP_E_INVAL;
+        }
+        P_hi = g->n_P ? g->P[g->n_P - 1] : 2;
+    } else {
+        if (g->P_lo < 2 || g->P_hi < g->P_lo) return PLOGP_E_INVAL;
+        P_hi = g->P_hi;
+    }
+    for (int i = 0; i < g->n_m; ++i) {
+        const uint64_t m = g->m[i];
+        if (m == 0 || m % g->dtype_bytes) return PLOGP_E_INVAL;
+        if (i && m <= g->m[i - 1]) return PLOGP_E_INVAL;
+        if (m >= kTwo32) return PLOGP_E_RANGE;
+    }
+    if (g->n_m > 0 && double(P_hi) * double(g->m[g->n_m - 1]) >= kTwo53) return PLOGP_E_RANGE;
+    int64_t n_s = 0;
+    if (g->strategy_mask & kSegBits) {
+        if (g->s) {
+            if (g->n_s < 0) return PLOGP_E_INVAL;
+            for (int64_t i = 0; i < g->n_s; ++i) {
+                const uint64_t s = g->s[i];
+                if (s == 0 || s % g->dtype_bytes) return PLOGP_E_INVAL;
+                if (i && s <= g->s[i - 1]) return PLOGP_E_INVAL;
+                if (s >= kTwo32) return PLOGP_E_RANGE;
+            }
+            n_s = g->n_s;
+        } else {
+            if (g->s_step == 0 || g->s_step % g->dtype_bytes) return PLOGP_E_INVAL;
+            if (g->s_lo == 0 || g->s_lo % g->dtype_bytes) return PLOGP_E_INVAL;
+            if (g->s_hi >= g->s_lo) {
+                if (g->s_hi >= kTwo32) return PLOGP_E_RANGE;
+                n_s = int64_t((g->s_hi - g->s_lo) / g->s_step) + 1;
+            }
+        }
+        if (n_s >= (int64_t(1) << 31)) return PLOGP_E_RANGE;
+    }
+    (void)h;
+    *n_s_out = n_s;
+    return PLOGP_OK;
+}
+
+// Builds (or reuses) the launch plan of a grid and makes its device arrays current.
+int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
+{
+    if (!g || g->n_m < 0 || (g->n_m > 0 && !g->m)) return PLOGP_E_INVAL;
+    if (g->P && g->n_P < 0) return PLOGP_E_INVAL;
+    if ((g->strategy_mask & kSegBits) && g->s && g->n_s < 0) return PLOGP_E_INVAL;
+    // ---- cache key: every input that the plan depends on ----
+    std::vector<unsigned char> key;
+    key.reserve(256 + size_t(std::max(g->n_m, 0)) * 8);
+    const int has_P = g->P != nullptr, has_s = g->s != nullptr;
+    put(key, has_P);
+    if (has_P) { put(key, g->n_P); put_array(key, g->P, size_t(std::max(g->n_P, 0))); }
+    else { put(key, g->P_lo); put(key, g->P_hi); }
+    put(key, g->n_m);
+    put_array(key, g->m, size_t(std::max(g->n_m, 0)));
+    put(key, g->strategy_mask); put(key, g->k_mode); put(key, g->dtype_bytes);
+    if (g->strategy_mask & kSegBits) {
+        put(key, has_s);
+        if (has_s) { put(key, g->n_s); put_array(key, g->s, size_t(std::max<int64_t>(g->n_s, 0))); }
+        else { put(key, g->s_lo); put(key, g->s_hi); put(key, g->s_step); }
+    }
+    if (!h->plan.key.empty() && h->plan.key == key) return PLOGP_OK;
+
+    int64_t n_s64 = 0;
+    int rc = validate_grid(h, g, &n_s64);
+    if (rc != PLOGP_OK) return rc;
+
+    Plan pl;
+    pl.key = std::move(key);
+    const int n_P = g->P ? g->n_P : (g->P_hi - g->P_lo + 1);
+    const int n_m = g->n_m;
+    const int n_s = int(n_s64);
+    pl.empty = (n_P == 0 || n_m == 0 || g->strategy_mask == 0);
+    if (pl.empty) { h->plan = std::move(pl); return PLOGP_OK; }
+
+    const int64_t P_hi = g->P ? g->P[n_P - 1] : g->P_hi;
+    pl.n_seg = __builtin_popcount(g->strategy_mask & kSegBits);
+    pl.inline_sweep = pl.n_seg == 0 || n_s <= kMaxInlineS;
+
+    // candidates per message size (grid values s <= m)
+    std::vector<int32_t> ns_of_m(n_m, 0);
+    int ns_max = 0;
+    if (pl.n_seg) {
+        for (int i = 0; i < n_m; ++i) {
+            const uint64_t m = g->m[i];
+            int64_t c;
+            if (g->s) c = std::upper_bound(g->s, g->s + n_s, m) - g->s;
+            else {
+                const uint64_t top = std::min<uint64_t>(m, g->s_hi);
+                c = (n_s > 0 && top >= g->s_lo) ? int64_t((top - g->s_lo) / g->s_step) + 1 : 0;
+            }
+            ns_of_m[i] = int32_t(c);
+            ns_max = std::max(ns_max, int(c));
+        }
+    }
+
+    // ---- fused kernel tiling ----
+    const int pass_P = kWarps * kFusedR;
+    const int total_passes = (n_P + pass_P - 1) / pass_P;
+    pl.n_mtiles = (n_m + 31) / 32;
+    const long long base_blocks = (long long)pl.n_mtiles * h->T.n_tables;
+    const long long target = (long long)h->sm_count * 8;
+    int n_ptiles = 1;
+    if (base_blocks < target) n_ptiles = int(std::min<long long>(total_passes, (target + base_blocks - 1) / base_blocks));
+    n_ptiles = std::min(n_ptiles, 256);
+    pl.passes_per_tile = (total_passes + n_ptiles - 1) / n_ptiles;
+    pl.n_ptiles = (total_passes + pl.passes_per_tile - 1) / pl.passes_per_tile;
+
+    // ---- device arrays ----
+    std::vector<unsigned char> blob;
+    std::vector<uint32_t> m32(n_m);
+    for (int i = 0; i < n_m; ++i) m32[i] = uint32_t(g->m[i]);
+    const size_t off_m = append_aligned(blob, m32);
+    const size_t off_ns = append_aligned(blob, ns_of_m);
+    size_t off_P = 0, off_s = 0;
+    if (g->P) off_P = append_aligned(blob, std::vector<int32_t>(g->P, g->P + n_P));
+    if (pl.n_seg && g->s) {
+        std::vector<uint32_t> s32(n_s);
+        for (int i = 0; i < n_s; ++i) s32[i] = uint32_t(g->s[i]);
+        off_s = append_aligned(blob, s32);
+    }
+
+    // ---- sweep kernel plan: (m, chunk) pairs, heaviest first ----
+    if (!pl.inline_sweep) {
+        pl.chunk_len = std::max(2048, ((ns_max + 31) / 32 + kSweepSub - 1) / kSweepSub * kSweepSub);
+        std::vector<int32_t> pair_base(n_m + 1, 0);
+        struct Pair { int32_t m, chunk, row, len; };
+        std::vector<Pair> pairs;
+        for (int i = 0; i < n_m; ++i) {
+            pair_base[i] = int32_t(pairs.size());
+            for (int c = 0; c * pl.chunk_len < ns_of_m[i]; ++c)
+                pairs.push_back({i, c, int32_t(pairs.size()), std::min(pl.chunk_len, ns_of_m[i] - c * pl.chunk_len)});
+        }
+        pair_base[n_m] = int32_t(pairs.size());
+        pl.n_pairs = int(pairs.size());
+        std::stable_sort(pairs.begin(), pairs.end(), [](const Pair &a, const Pair &b) { return a.len > b.len; });
+        std::vector<int32_t> pm(pl.n_pairs), pc(pl.n_pairs), pr(pl.n_pairs);
+        for (int i = 0; i < pl.n_pairs; ++i) { pm[i] = pairs[i].m; pc[i] = pairs[i].chunk; pr[i] = pairs[i].row; }
+        pl.off_pair_m = append_aligned(blob, pm);
+        pl.off_pair_chunk = append_aligned(blob, pc);
+        pl.off_pair_row = append_aligned(blob, pr);
+        pl.off_pair_base = append_aligned(blob, pair_base);
+        pl.sweep_ptiles = (n_P + kThreads * kSweepR - 1) / (kThreads * kSweepR);
+    }
+
+    if (blob.size() > h->grid_cap) {
+        if (h->d_grid) CK(cudaFree(h->d_grid));
+        h->d_grid = nullptr;
+        h->grid_cap = 0;
+        const size_t cap = std::max<size_t>(blob.size() * 2, 4096);
+        CK(cudaMalloc(&h->d_grid, cap));
+        h->grid_cap = cap;
+    }
+    // The source is pageable host memory: the runtime stages it before returning.
+    CK(cudaMemcpyAsync(h->d_grid, blob.data(), blob.size(), cudaMemcpyHostToDevice, st));
+
+    GridDev &G = pl.G;
+    G.P_list = g->P ? reinterpret_cast<const int32_t *>(h->d_grid + off_P) : nullptr;
+    G.n_P = n_P;
+    G.P_lo = g->P ? 0 : g->P_lo;
+    G.m_list = reinterpret_cast<const uint32_t *>(h->d_grid + off_m);
+    G.n_m = n_m;
+    G.s_list = (pl.n_seg && g->s) ? reinterpret_cast<const uint32_t *>(h->d_grid + off_s) : nullptr;
+    G.n_s = pl.n_seg ? n_s : 0;
+    G.s_lo = uint32_t(g->s_lo);
+    G.s_step = uint32_t(g->s_step);
+    G.ns_of_m = reinterpret_cast<const int32_t *>(h->d_grid + off_ns);
+    G.mask = g->strategy_mask;
+    G.k_mode = g->k_mode;
+    G.lc_max = std::max(1, ceil_log2(P_hi));
+
+    // ---- scratch: sweep partials (per table batch) and Scatter Chain tile prefixes ----
+    const bool need_carry = ((g->strategy_mask >> 11) & 1u) && pl.n_ptiles > 1;
+    size_t per_table = 0;
+    if (!pl.inline_sweep) per_table += size_t(pl.n_seg) * pl.n_pairs * n_P * (sizeof(double) + sizeof(uint32_t)) + 64;
+    if (need_carry) per_table += size_t(pl.n_ptiles) * n_m * sizeof(double) + 64;
+    pl.tables_per_batch = h->T.n_tables;
+    if (!pl.inline_sweep && per_table * h->T.n_tables > kSweepScratchLimit)
+        pl.tables_per_batch = int(std::max<size_t>(1, kSweepScratchLimit / per_table));
+    pl.tables_per_batch = std::min(pl.tables_per_batch, 65535);
+    pl.scratch_bytes = per_table ? per_table * pl.tables_per_batch + 256 : 0;
+    if (pl.scratch_bytes > h->ws_cap) {
+        if (h->d_ws) CK(cudaFree(h->d_ws));
+        h->d_ws = nullptr;
+        h->ws_cap = 0;
+        cudaError_t e = cudaMalloc(&h->d_ws, pl.scratch_bytes);
+        if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return PLOGP_E_NOMEM; }
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(scratch)");
+        h->ws_cap = pl.scratch_bytes;
+    }
+    h->plan = std::move(pl);
+    return PLOGP_OK;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cudaStream_t st)
+{
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev != h->device) return PLOGP_E_INVAL;
+    int rc = prepare(h, g, st);
+    if (rc != PLOGP_OK) { h->plan = Plan(); return rc; }
+    const Plan &pl = h->plan;
+    if (pl.empty) return PLOGP_OK;
+    const bool s1 = (pl.G.mask >> 11) & 1u;
+    const bool need_carry = s1 && pl.n_ptiles > 1;
+
+    for (int t0 = 0; t0 < h->T.n_tables; t0 += pl.tables_per_batch) {
+        const int nt = std::min(pl.tables_per_batch, h->T.n_tables - t0);
+        unsigned char *ws = h->d_ws;
+        double *part_time = nullptr;
+        uint32_t *part_idx = nullptr;
+        double *tile_sum = nullptr;
+        if (!pl.inline_sweep) {
+            const size_t cells = size_t(nt) * pl.n_seg * pl.n_pairs * pl.G.n_P;
+            part_time = reinterpret_cast<double *>(ws);
+            ws += align_up(cells * sizeof(double), 256);
+            part_idx = reinterpret_cast<uint32_t *>(ws);
+            ws += align_up(cells * sizeof(uint32_t), 256);
+        }
+        if (need_carry) tile_sum = reinterpret_cast<double *>(ws);
+
+        if (!pl.inline_sweep && pl.n_pairs > 0) {
+            SweepParams sp{};
+            sp.T = h->T; sp.G = pl.G;
+            sp.pair_m = reinterpret_cast<const int32_t *>(h->d_grid + pl.off_pair_m);
+            sp.pair_chunk = reinterpret_cast<const int32_t *>(h->d_grid + pl.off_pair_chunk);
+            sp.pair_row = reinterpret_cast<const int32_t *>(h->d_grid + pl.off_pair_row);
+            sp.n_pairs = pl.n_pairs; sp.n_ptiles = pl.sweep_ptiles; sp.chunk_len = pl.chunk_len;
+            sp.part_time = part_time; sp.part_idx = part_idx; sp.n_seg = pl.n_seg; sp.table0 = t0;
+            CK(launch_sweep(sp, nt, st));
+        }
+        if (need_carry) {
+            S1Params s{};
+            s.T = h->T; s.G = pl.G;
+            s.n_mtiles = pl.n_mtiles; s.n_ptiles = pl.n_ptiles; s.passes_per_tile = pl.passes_per_tile;
+            s.table0 = t0; s.n_tables_launch = nt; s.tile_sum = tile_sum;
+            CK(launch_s1_tiles(s, st));
+        }
+        FusedParams fp = out;
+        fp.T = h->T; fp.G = pl.G;
+        fp.n_mtiles = pl.n_mtiles; fp.n_ptiles = pl.n_ptiles; fp.passes_per_tile = pl.passes_per_tile;
+        fp.table0 = t0; fp.n_tables_launch = nt;
+        fp.s1_carry = tile_sum;
+        // part_time doubles as the "segmented minima come from the sweep kernel" switch
+        fp.part_time = pl.inline_sweep ? nullptr : part_time;
+        fp.part_idx = part_idx;
+        fp.pair_base = pl.inline_sweep ? nullptr : reinterpret_cast<const int32_t *>(h->d_grid + pl.off_pair_base);
+        fp.n_pairs = pl.n_pairs; fp.n_seg = pl.n_seg;
+        CK(launch_fused(fp, predict, st));
+    }
+    return PLOGP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int plogp_table_load(int n_tables, int n_bp, const uint64_t *sizes_bytes, int sizes_shared,
+                     const double *gap, const double *latency, plogp_tables **out)
+{
+    if (!sizes_bytes || !gap || !latency || !out) return PLOGP_E_INVAL;
+    if (n_tables < 1 || n_bp < 2) return PLOGP_E_INVAL;
+    if (n_bp > PLOGP_MAX_BREAKPOINTS) return PLOGP_E_RANGE;
+    int npad = 2;
+    while (npad < n_bp - 1) npad <<= 1;
+
+    std::vector<double> tab, lat;
+    try {
+        tab.assign(size_t(n_tables) * 3 * npad, 0.0);
+        lat.assign(latency, latency + n_tables);
+    } catch (const std::bad_alloc &) { return PLOGP_E_NOMEM; }
+
+    const double inf = std::numeric_limits<double>::infinity();
+    for (int t = 0; t < n_tables; ++t) {
+        const uint64_t *sz = sizes_bytes + (sizes_shared ? 0 : size_t(t) * n_bp);
+        const double *gp = gap + size_t(t) * n_bp;
+        if (!std::isfinite(lat[t]) || lat[t] < 0.0) return PLOGP_E_INVAL;
+        for (int i = 0; i < n_bp; ++i) {
+            if (!std::isfinite(gp[i]) || gp[i] < 0.0) return PLOGP_E_INVAL;
+            if (i && sz[i] <= sz[i - 1]) return PLOGP_E_INVAL;
+            if (double(sz[i]) >= kTwo53) return PLOGP_E_RANGE;
+        }
+        double *key = tab.data() + size_t(t) * 3 * npad, *g0 = key + npad, *sl = g0 + npad;
+        for (int i = 0; i < npad; ++i) {
+            if (i <= n_bp - 2) {
+                key[i] = double(sz[i]);
+                g0[i] = gp[i];
+                sl[i] = (gp[i + 1] - gp[i]) / double(sz[i + 1] - sz[i]);
+            } else {
+                key[i] = inf;
+                g0[i] = 0.0;
+                sl[i] = 0.0;
+            }
+        }
+    }
+
+    plogp_tables *h = new (std::nothrow) plogp_tables();
+    if (!h) return PLOGP_E_NOMEM;
+    auto fail = [&](int rc) { plogp_table_free(h); return rc; };
+    cudaError_t e;
+    if ((e = cudaGetDevice(&h->device)) != cudaSuccess) return fail(cuda_fail(e, "cudaGetDevice"));
+    if ((e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device)) != cudaSuccess)
+        return fail(cuda_fail(e, "cudaDeviceGetAttribute"));
+    if ((e = cudaMalloc(&h->d_tab, tab.size() * sizeof(double))) != cudaSuccess)
+        return fail(e == cudaErrorMemoryAllocation ? (cudaGetLastError(), PLOGP_E_NOMEM) : cuda_fail(e, "cudaMalloc(tables)"));
+    if ((e = cudaMalloc(&h->d_lat, lat.size() * sizeof(double))) != cudaSuccess)
+        return fail(e == cudaErrorMemoryAllocation ? (cudaGetLastError(), PLOGP_E_NOMEM) : cuda_fail(e, "cudaMalloc(latency)"));
+    if ((e = cudaMemcpy(h->d_tab, tab.data(), tab.size() * sizeof(double), cudaMemcpyHostToDevice)) != cudaSuccess)
+        return fail(cuda_fail(e, "cudaMemcpy(tables)"));
+    if ((e = cudaMemcpy(h->d_lat, lat.data(), lat.size() * sizeof(double), cudaMemcpyHostToDevice)) != cudaSuccess)
+        return fail(cuda_fail(e, "cudaMemcpy(latency)"));
+    h->T.tab = h->d_tab;
+    h->T.lat = h->d_lat;
+    h->T.n_tables = n_tables;
+    h->T.n_bp = n_bp;
+    h->T.npad = npad;
+    *out = h;
+    return PLOGP_OK;
+}
+
+int plogp_table_free(plogp_tables *h)
+{
+    if (!h) return PLOGP_OK;
+    int rc = PLOGP_OK;
+    void *bufs[] = {h->d_tab, h->d_lat, h->d_grid, h->d_ws};
+    for (void *b : bufs) {
+        if (b) {
+            cudaError_t e = cudaFree(b);
+            if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree");
+        }
+    }
+    delete h;
+    return rc;
+}
+
+int plogp_predict(plogp_tables *tables, const plogp_grid *grid, double *d_time, uint32_t *d_best_s, void *stream)
+{
+    if (!tables || !grid || !d_time) return PLOGP_E_INVAL;
+    FusedParams out{};
+    out.p_time = d_time;
+    out.p_best_s = d_best_s;
+    return run(tables, grid, true, out, static_cast<cudaStream_t>(stream));
+}
+
+int plogp_select_best(plogp_tables *tables, const plogp_grid *grid, uint8_t *d_strategy, uint32_t *d_s_bytes,
+                      double *d_time, void *stream)
+{
+    if (!tables || !grid || !d_strategy || !d_s_bytes || !d_time) return PLOGP_E_INVAL;
+    FusedParams out{};
+    out.d_strategy = d_strategy;
+    out.d_sbytes = d_s_bytes;
+    out.d_time = d_time;
+    return run(tables, grid, false, out, static_cast<cudaStream_t>(stream));
+}
+
+const char *plogp_status_string(int status)
+{
+    switch (status) {
+    case PLOGP_OK: return "ok";
+    case PLOGP_E_INVAL: return "invalid argument";
+    case PLOGP_E_NOMEM: return "out of memory";
+    case PLOGP_E_CUDA: return "CUDA runtime error";
+    case PLOGP_E_RANGE: return "value out of the supported range";
+    default: return "unknown status";
+    }
+}
+
+const char *plogp_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+double plogp_fp64_fma_rate(double milliseconds)
+{
+    if (!(milliseconds > 0.0)) return double(PLOGP_E_INVAL);
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return double(PLOGP_E_CUDA);
+    double *sink = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    double rate = double(PLOGP_E_CUDA);
+    const int blocks = sms * 8;
+    const double fma_per_iter = double(blocks) * kThreads * 32.0;
+    do {
+        if (cudaMalloc(&sink, sizeof(double)) != cudaSuccess) break;
+        if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) break;
+        int iters = 2000;
+        float ms = 0.f;
+        bool ok = true;
+        for (int round = 0; round < 3 && ok; ++round) {  // warm-up, calibration, measurement
+            ok = cudaEventRecord(e0) == cudaSuccess && launch_fp64_probe(sink, iters, blocks, nullptr) == cudaSuccess &&
+                 cudaEventRecord(e1) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess &&
+                 cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess;
+            if (ok && round == 1 && ms > 0.f) iters = int(std::min(2e8, std::max(2000.0, iters * milliseconds / ms)));
+        }
+        if (ok && ms > 0.f) rate = fma_per_iter * iters / (ms * 1e-3);
+    } while (0);
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (sink) cudaFree(sink);
+    return rate;
+}
+
+}  // extern "C"

@@ -1,0 +1,91 @@
+// Internal declarations shared by the host side (api.cu) and the kernels (kernels.cu).
+// Nothing here is part of the public ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace plogp {
+
+// Tables as they live in device memory.  Per table: three runs of `npad` doubles
+//   key[npad]   breakpoint sizes usable as interval starts (index <= n_bp-2), +inf beyond
+//   gap[npad]   g at the interval start
+//   slope[npad] (g[i+1]-g[i]) / (size[i+1]-size[i])
+// npad is a power of two >= n_bp-1, so the interval search needs no bounds checks.
+struct TableDev {
+    const double *tab;  // [n_tables][3*npad]
+    const double *lat;  // [n_tables]
+    int n_tables, n_bp, npad;
+};
+
+struct GridDev {
+    const int32_t *P_list;  // device [n_P] or nullptr => P = P_lo + index
+    int n_P, P_lo;
+    const uint32_t *m_list;  // device [n_m]
+    int n_m;
+    const uint32_t *s_list;  // device [n_s] or nullptr => s = s_lo + index * s_step
+    int n_s;
+    uint32_t s_lo, s_step;
+    const int32_t *ns_of_m;  // device [n_m]: number of candidates s <= m (0 => unsegmented fallback)
+    uint32_t mask;
+    int k_mode;
+    int lc_max;  // ceil(log2 P_hi)
+};
+
+// Segment-sweep kernel (large candidate lists): partial minima per (table, segmented strategy,
+// (m, chunk) pair, P).
+struct SweepParams {
+    TableDev T;
+    GridDev G;
+    const int32_t *pair_m;      // device [n_pairs] in launch order (heaviest first)
+    const int32_t *pair_chunk;  // device [n_pairs]
+    const int32_t *pair_row;    // device [n_pairs]: row id of the pair (= pair_base[m] + chunk)
+    int n_pairs, n_ptiles, chunk_len;
+    double *part_time;   // [n_tables_batch][n_seg][n_pairs][n_P]
+    uint32_t *part_idx;  // same shape: index of s in the candidate list
+    int n_seg;           // enabled segmented strategies (slots in id order)
+    int table0;          // first table of this launch (blockIdx.y is relative to it)
+};
+
+struct FusedParams {
+    TableDev T;
+    GridDev G;
+    int n_mtiles, n_ptiles, passes_per_tile;  // a pass covers kWarps*R process counts
+    int table0, n_tables_launch;
+    const double *s1_carry;  // [n_tables_launch][n_ptiles][n_m] exclusive tile prefixes, or nullptr
+    // segmented minima precomputed by the sweep kernel (nullptr => inline sweep)
+    const double *part_time;
+    const uint32_t *part_idx;
+    const int32_t *pair_base;  // device [n_m+1]
+    int n_pairs, n_seg;
+    // outputs: decision table
+    uint8_t *d_strategy;
+    uint32_t *d_sbytes;
+    double *d_time;
+    // outputs: predicted planes
+    double *p_time;
+    uint32_t *p_best_s;
+};
+
+struct S1Params {
+    TableDev T;
+    GridDev G;
+    int n_mtiles, n_ptiles, passes_per_tile;
+    int table0, n_tables_launch;
+    double *tile_sum;  // [n_tables_launch][n_ptiles][n_m]
+};
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kFusedR = 4;   // process counts per thread and pass in the fused kernel
+constexpr int kSweepR = 8;   // process counts per thread in the sweep kernel
+constexpr int kSweepSub = 256;  // candidates staged per sub-chunk
+constexpr int kMaxInlineS = 64;
+
+size_t fused_smem_bytes(const TableDev &T, const GridDev &G, bool inline_sweep);
+cudaError_t launch_fused(const FusedParams &p, bool predict, cudaStream_t st);
+cudaError_t launch_sweep(const SweepParams &p, int n_tables_launch, cudaStream_t st);
+cudaError_t launch_s1_tiles(const S1Params &p, cudaStream_t st);
+cudaError_t launch_fp64_probe(double *d_sink, int iters, int blocks, cudaStream_t st);
+
+}  // namespace plogp

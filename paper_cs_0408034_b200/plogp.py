@@ -1,0 +1,226 @@
+"""Python binding of the C ABI in ``include/plogp.h`` (same names, argument marshalling only).
+
+Every step of the evaluation runs in the CUDA library; torch is used for device memory and the
+current stream.  There is no fallback: if the shared object is missing, importing this module
+raises, and the calls need a CUDA device.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libplogp.so")
+
+N_STRATEGIES = 13
+SEGMENTED_IDS = (2, 5, 9)
+EXPORTS = ("plogp_table_load", "plogp_table_free", "plogp_predict", "plogp_select_best",
+           "plogp_status_string", "plogp_last_cuda_error", "plogp_fp64_fma_rate")
+
+OK, E_INVAL, E_NOMEM, E_CUDA, E_RANGE = 0, -1, -2, -3, -4
+
+
+class Grid(C.Structure):
+    """Mirror of ``plogp_grid``."""
+    _fields_ = [("P", C.POINTER(C.c_int32)), ("n_P", C.c_int32), ("P_lo", C.c_int32), ("P_hi", C.c_int32),
+                ("m", C.POINTER(C.c_uint64)), ("n_m", C.c_int32),
+                ("s", C.POINTER(C.c_uint64)), ("n_s", C.c_int64),
+                ("s_lo", C.c_uint64), ("s_hi", C.c_uint64), ("s_step", C.c_uint64),
+                ("dtype_bytes", C.c_uint32), ("strategy_mask", C.c_uint32), ("k_mode", C.c_int32)]
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError("%s is missing: build it with `python __graft_entry__.py` (nvcc, sm_100a); "
+                      "there is no CPU fallback" % LIB_PATH)
+lib = C.CDLL(LIB_PATH)
+for _name in EXPORTS:
+    if not hasattr(lib, _name):
+        raise ImportError("%s does not export %s" % (LIB_PATH, _name))
+
+lib.plogp_table_load.restype = C.c_int
+lib.plogp_table_load.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
+                                 C.POINTER(C.c_void_p)]
+lib.plogp_table_free.restype = C.c_int
+lib.plogp_table_free.argtypes = [C.c_void_p]
+lib.plogp_predict.restype = C.c_int
+lib.plogp_predict.argtypes = [C.c_void_p, C.POINTER(Grid), C.c_void_p, C.c_void_p, C.c_void_p]
+lib.plogp_select_best.restype = C.c_int
+lib.plogp_select_best.argtypes = [C.c_void_p, C.POINTER(Grid), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+lib.plogp_status_string.restype = C.c_char_p
+lib.plogp_status_string.argtypes = [C.c_int]
+lib.plogp_last_cuda_error.restype = C.c_char_p
+lib.plogp_last_cuda_error.argtypes = []
+lib.plogp_fp64_fma_rate.restype = C.c_double
+lib.plogp_fp64_fma_rate.argtypes = [C.c_double]
+
+
+class PlogpError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = "%s: %s" % (where, lib.plogp_status_string(status).decode())
+        if status == E_CUDA:
+            msg += " [%s]" % lib.plogp_last_cuda_error().decode()
+        super().__init__(msg)
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise PlogpError(status, where)
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data
+
+
+class Tables:
+    """Owner of a ``plogp_tables`` handle (pLogP parameter sets on the current device)."""
+
+    def __init__(self, sizes, gaps, latency):
+        sizes = np.ascontiguousarray(sizes, dtype=np.uint64)
+        gaps = np.ascontiguousarray(gaps, dtype=np.float64)
+        latency = np.ascontiguousarray(latency, dtype=np.float64)
+        if gaps.ndim != 2 or latency.shape != (gaps.shape[0],):
+            raise ValueError("gaps must be [n_tables][n_bp] and latency [n_tables]")
+        shared = sizes.ndim == 1
+        if sizes.shape != (gaps.shape[1],) and sizes.shape != gaps.shape:
+            raise ValueError("sizes must be [n_bp] or [n_tables][n_bp]")
+        self.n_tables, self.n_bp = int(gaps.shape[0]), int(gaps.shape[1])
+        h = C.c_void_p()
+        _check(lib.plogp_table_load(self.n_tables, self.n_bp, _ptr(sizes), int(shared), _ptr(gaps),
+                                    _ptr(latency), C.byref(h)), "plogp_table_load")
+        self._h = h
+
+    @classmethod
+    def from_workload(cls, w) -> "Tables":
+        return cls(w.sizes, w.gaps, w.latency)
+
+    @property
+    def handle(self):
+        if self._h is None:
+            raise ValueError("tables were freed")
+        return self._h
+
+    def free(self) -> None:
+        if getattr(self, "_h", None) is not None:
+            h, self._h = self._h, None
+            _check(lib.plogp_table_free(h), "plogp_table_free")
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.free()
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+class GridArgs:
+    """Keeps the host arrays of a ``plogp_grid`` alive next to the struct."""
+
+    def __init__(self, m, P=None, P_lo=2, P_hi=2, s=None, s_lo=0, s_hi=0, s_step=0,
+                 dtype_bytes=4, strategy_mask=(1 << 13) - 1, k_mode=0):
+        self.m = np.ascontiguousarray(m, dtype=np.uint64)
+        self.P = None if P is None else np.ascontiguousarray(P, dtype=np.int32)
+        self.s = None if s is None else np.ascontiguousarray(s, dtype=np.uint64)
+        g = Grid()
+        if self.P is not None:
+            g.P = self.P.ctypes.data_as(C.POINTER(C.c_int32))
+            g.n_P = len(self.P)
+        g.P_lo, g.P_hi = int(P_lo), int(P_hi)
+        g.m = self.m.ctypes.data_as(C.POINTER(C.c_uint64))
+        g.n_m = len(self.m)
+        if self.s is not None:
+            g.s = self.s.ctypes.data_as(C.POINTER(C.c_uint64))
+            g.n_s = len(self.s)
+        g.s_lo, g.s_hi, g.s_step = int(s_lo), int(s_hi), int(s_step)
+        g.dtype_bytes, g.strategy_mask, g.k_mode = int(dtype_bytes), int(strategy_mask), int(k_mode)
+        self.struct = g
+
+    @classmethod
+    def from_workload(cls, w) -> "GridArgs":
+        return cls(w.m, None, w.P_lo, w.P_hi, w.s_list, w.s_lo, w.s_hi, w.s_step, w.dtype_bytes,
+                   w.strategy_mask, w.k_mode)
+
+    @property
+    def n_P(self) -> int:
+        return len(self.P) if self.P is not None else self.struct.P_hi - self.struct.P_lo + 1
+
+    @property
+    def n_m(self) -> int:
+        return len(self.m)
+
+    @property
+    def ref(self):
+        return C.byref(self.struct)
+
+
+def _as_grid(grid) -> GridArgs:
+    return grid if isinstance(grid, GridArgs) else GridArgs.from_workload(grid)
+
+
+def _stream_ptr(stream) -> int:
+    import torch
+    st = torch.cuda.current_stream() if stream is None else stream
+    return int(st.cuda_stream)
+
+
+@dataclass
+class Prediction:
+    time: "object"    # torch.float64 [n_tables][13][n_P][n_m]
+    best_s: "object"  # torch.int32 (uint32 bit pattern) [n_tables][3][n_P][n_m]
+
+
+@dataclass
+class DecisionTable:
+    strategy: "object"  # torch.uint8 [n_tables][2][n_P][n_m]
+    s_bytes: "object"   # torch.int32 (uint32 bit pattern) [n_tables][2][n_P][n_m]
+    time: "object"      # torch.float64 [n_tables][2][n_P][n_m]
+
+
+def predict(tables: Tables, grid, out: Optional[Prediction] = None, stream=None, want_best_s: bool = True) -> Prediction:
+    """``plogp_predict``: all enabled models of Table 1 / Table 2, segmented ones reduced over s."""
+    import torch
+    g = _as_grid(grid)
+    if out is None:
+        shape = (tables.n_tables, N_STRATEGIES, g.n_P, g.n_m)
+        time = torch.full(shape, float("nan"), dtype=torch.float64, device="cuda")
+        best = torch.zeros((tables.n_tables, 3, g.n_P, g.n_m), dtype=torch.int32, device="cuda") if want_best_s else None
+        out = Prediction(time, best)
+    _check(lib.plogp_predict(tables.handle, g.ref, out.time.data_ptr(),
+                             None if out.best_s is None else out.best_s.data_ptr(), _stream_ptr(stream)),
+           "plogp_predict")
+    return out
+
+
+def alloc_decision(n_tables: int, n_P: int, n_m: int) -> DecisionTable:
+    import torch
+    shape = (n_tables, 2, n_P, n_m)
+    return DecisionTable(torch.full(shape, 255, dtype=torch.uint8, device="cuda"),
+                         torch.zeros(shape, dtype=torch.int32, device="cuda"),
+                         torch.full(shape, float("nan"), dtype=torch.float64, device="cuda"))
+
+
+def select_best(tables: Tables, grid, out: Optional[DecisionTable] = None, stream=None) -> DecisionTable:
+    """``plogp_select_best``: best strategy, its segment size and predicted time per (collective, P, m)."""
+    g = _as_grid(grid)
+    if out is None:
+        out = alloc_decision(tables.n_tables, g.n_P, g.n_m)
+    _check(lib.plogp_select_best(tables.handle, g.ref, out.strategy.data_ptr(), out.s_bytes.data_ptr(),
+                                 out.time.data_ptr(), _stream_ptr(stream)), "plogp_select_best")
+    return out
+
+
+def fp64_fma_rate(milliseconds: float = 50.0) -> float:
+    """``plogp_fp64_fma_rate``: sustained thread-level DFMA instructions per second on this device."""
+    r = lib.plogp_fp64_fma_rate(float(milliseconds))
+    if r < 0:
+        raise PlogpError(int(r), "plogp_fp64_fma_rate")
+    return r

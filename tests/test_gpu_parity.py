@@ -1,0 +1,133 @@
+"""GPU results through the C ABI against the CPU oracle, element by element, on seeded workloads
+shaped like the five benchmark configurations (reduced where the oracle would take too long) plus
+edge cases.  Tolerances: see tests/parity.py."""
+import numpy as np
+import pytest
+
+from paper_cs_0408034_b200 import workloads as wl
+from parity import check_decision, check_prediction, oracle_tables
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def plogp():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_cs_0408034_b200 import plogp as mod
+    return mod
+
+
+def run_both(plogp, w, **sub):
+    import torch
+    ot = oracle_tables(w)
+    with plogp.Tables.from_workload(w) as tabs:
+        dec = plogp.select_best(tabs, w)
+        pred = plogp.predict(tabs, w)
+        torch.cuda.synchronize()
+        n = check_decision(w, ot, dec, **sub) + check_prediction(w, ot, pred, **sub)
+    assert n > 0
+    return dec, pred
+
+
+def test_config1_full(plogp):
+    run_both(plogp, wl.config1())
+
+
+def test_config1_all_strategies_and_floor_mode(plogp):
+    from dataclasses import replace
+    w = replace(wl.config1(), strategy_mask=wl.ALL_STRATEGIES)
+    run_both(plogp, w)
+    run_both(plogp, replace(w, k_mode=1))
+
+
+def test_config2_full_size(plogp):
+    # 1023 x 256 cells x 13 strategies, 64 candidates: the oracle needs a few seconds
+    run_both(plogp, wl.config2())
+
+
+def test_config2_ragged_tiles(plogp):
+    # n_m = 37 (one full tile + ragged tail), n_P = 77 (ragged pass), 13 candidates
+    run_both(plogp, wl.config2(P_hi=78, n_m=37, n_s=13))
+
+
+def test_config3_reduced_goes_through_the_sweep_kernel(plogp):
+    # candidates = every multiple of 4 up to 64 KB (16384 > inline limit): chunks, several P tiles' worth of lanes
+    w = wl.config3(P_hi=300, n_m=10, m_lo=4 << 10, m_hi=1 << 18, s_hi=1 << 16)
+    run_both(plogp, w)
+
+
+def test_config3_sweep_with_all_segmented_strategies(plogp):
+    from dataclasses import replace
+    w = replace(wl.config3(P_hi=2200, n_m=5, m_lo=1 << 10, m_hi=1 << 15, s_hi=1 << 13), strategy_mask=wl.ALL_STRATEGIES)
+    run_both(plogp, w, p_idx=np.r_[0:40, 1000:1040, 2040:2060, 2190:2199])
+    for mask in (1 << 2, 1 << 9, (1 << 2) | (1 << 9), (1 << 5) | (1 << 9)):
+        run_both(plogp, replace(w, strategy_mask=mask, P_hi=130))
+
+
+def test_config4_reduced_batch(plogp):
+    w = wl.config4(n_tables=6)
+    run_both(plogp, w, tables=[0, 3, 5], p_idx=np.r_[0:70, 250:260, 500:511])
+
+
+def test_config5_reduced_long_scan(plogp):
+    # P up to 9000: several P tiles, exercises the tile-sum / tile-scan carry of the Scatter Chain
+    run_both(plogp, wl.config5(P_hi=9000, n_m=40))
+
+
+def test_config5_full_size_sampled_rows(plogp):
+    import torch
+    w = wl.config5()
+    ot = oracle_tables(w)
+    with plogp.Tables.from_workload(w) as tabs:
+        dec = plogp.select_best(tabs, w)
+        pred = plogp.predict(tabs, w, want_best_s=False)
+        torch.cuda.synchronize()
+        p_idx = np.unique(np.r_[0:64, 4090:4100, 32760:32775, 65500:65535, np.arange(0, 65535, 997)])
+        m_idx = np.array([0, 1, 31, 32, 63])
+        check_decision(w, ot, dec, p_idx=p_idx, m_idx=m_idx)
+        check_prediction(w, ot, pred, p_idx=p_idx, m_idx=m_idx)
+
+
+def test_explicit_P_list_with_gaps(plogp):
+    import torch
+    w = wl.config1()
+    P = np.array([2, 3, 4, 8, 9, 16, 17, 31, 32, 33, 50, 400, 1000], dtype=np.int32)
+    g = plogp.GridArgs(w.m, P=P, s=w.s_list, strategy_mask=wl.ALL_STRATEGIES)
+    from oracle import plogp_oracle as po
+    ot = oracle_tables(w)[0]
+    with plogp.Tables.from_workload(w) as tabs:
+        pred = plogp.predict(tabs, g)
+        torch.cuda.synchronize()
+    o = po.predict_grid(ot, wl.ALL_STRATEGIES, P, w.m, po.SGrid(w.s_list))
+    got = pred.time[0].cpu().numpy()
+    assert np.max(np.abs(got - o.time) / o.time) <= 1e-12
+    assert (pred.best_s[0].cpu().numpy().view(np.uint32) == o.best_s).all()
+
+
+def test_deterministic_across_runs(plogp):
+    import torch
+    w = wl.config2(P_hi=300, n_m=70, n_s=40)
+    with plogp.Tables.from_workload(w) as tabs:
+        a = plogp.select_best(tabs, w)
+        b = plogp.select_best(tabs, w)
+        torch.cuda.synchronize()
+    assert torch.equal(a.strategy, b.strategy) and torch.equal(a.s_bytes, b.s_bytes)
+    assert torch.equal(a.time.view(torch.int64), b.time.view(torch.int64))
+
+
+def test_single_cell_and_two_breakpoints(plogp):
+    import torch
+    from oracle import plogp_oracle as po
+    sizes = np.array([4, 1024], dtype=np.uint64)
+    gaps = np.array([[2.0, 12.0]])
+    with plogp.Tables(sizes, gaps, np.array([3.0])) as tabs:
+        g = plogp.GridArgs([512], P_lo=7, P_hi=7, s=[4, 64, 512, 1024])
+        pred = plogp.predict(tabs, g)
+        dec = plogp.select_best(tabs, g)
+        torch.cuda.synchronize()
+    t = po.Table(sizes, gaps[0], 3.0)
+    o = po.predict_grid(t, wl.ALL_STRATEGIES, [7], [512], po.SGrid([4, 64, 512, 1024]))
+    np.testing.assert_allclose(pred.time[0, :, 0, 0].cpu().numpy(), o.time[:, 0, 0], rtol=1e-12)
+    od = po.select_grid(wl.ALL_STRATEGIES, o)
+    assert dec.strategy[0, :, 0, 0].tolist() == od.strategy[:, 0, 0].tolist()
