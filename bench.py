@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Benchmark of the pLogP tuner on N GPUs of one node (one process per GPU).
+
+A step is one pass of the whole path — plogp_select_best over the workload: table staging, g()
+interpolation, all enabled Table 1 / Table 2 models, the segment-size search, the Scatter sums,
+strategy selection and the decision-table stores.  The default workload is the batched
+multi-network configuration (4096 seeded tables x P = 2..512 x 128 m x 32 s, all 13 strategies);
+`--workload cfg3` times the exhaustive segment sweep instead.  With N > 1 every rank evaluates
+its own 4096 tables (different seeds): weak scaling, no data-path collective.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample of
+the same workload instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_cs_0408034_b200 import workloads as wl  # noqa: E402
+
+NOMINAL_FP64_FMA_RATE = 148 * 64 * 1.965e9  # SMs x FP64 lanes per SM x max SM clock
+FALLBACK_HBM_GBS = 6650.0
+
+
+def make_workload(name: str, scale: str, rank: int):
+    if name == "cfg4":
+        if scale == "small":
+            return wl.config4(n_tables=256, seed_offset=1000 * rank)
+        return wl.config4(seed_offset=1000 * rank)
+    if name == "cfg3":
+        if scale == "small":
+            return wl.config3(n_m=8, m_lo=256 << 10, m_hi=2 << 20, s_hi=256 << 10)
+        return wl.config3()
+    if name == "cfg2":
+        return wl.config2()
+    if name == "cfg5":
+        return wl.config5()
+    if name == "cfg1":
+        return wl.config1()
+    raise SystemExit("unknown workload %s" % name)
+
+
+def work_counts(w):
+    """Cells and the algorithmic work of one step (per segmented cell one DFMA and
+    one compare, per unsegmented cell one DFMA; bytes = the decision table written once)."""
+    mask = w.strategy_mask
+    n_seg = sum((mask >> b) & 1 for b in (2, 5, 9))
+    n_unseg = sum((mask >> b) & 1 for b in range(13)) - n_seg
+    seg_cells = w.n_tables * w.n_P * n_seg * int(w.n_candidates().sum())
+    unseg_cells = w.n_tables * w.n_P * n_unseg * w.n_m
+    dec = w.decision_cells()
+    return {"model_cells": seg_cells + unseg_cells, "segmented_cells": seg_cells, "decision_cells": dec,
+            "fp64_slots": 2 * seg_cells + unseg_cells, "hbm_bytes": 13 * dec}
+
+
+class ClockSampler:
+    """Samples SM clock, power and throttle reasons of one GPU through NVML while a region runs."""
+
+    def __init__(self, uuid: str, period_s: float = 0.02):
+        self.samples, self._stop, self._thread, self.sm_max, self.err = [], threading.Event(), None, None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            self.sm_max = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:  # NVML missing: report it instead of clocks
+            self.nv, self.err = None, repr(e)
+        self.period = period_s
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append((nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM),
+                                     nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0,
+                                     nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)))
+            except Exception as e:
+                self.err = repr(e)
+                return
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "error": self.err or "no samples"}
+        nv = self.nv
+        names = {"sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap, "hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksEventReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksEventReasonSwThermalSlowdown,
+                 "hw_power_brake": nv.nvmlClocksEventReasonHwPowerBrakeSlowdown}
+        seen = 0
+        for _, _, r in self.samples:
+            seen |= r
+        return {"sm_mhz": statistics.median(s[0] for s in self.samples), "sm_max_mhz": self.sm_max,
+                "reasons": [k for k, bit in names.items() if seen & bit],
+                "power_w_max": max(s[1] for s in self.samples), "samples": len(self.samples)}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return json.load(open(p)).get("hbm_gbs", FALLBACK_HBM_GBS), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def oracle_sample_rate(w, budget_s: float):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: whole tables for the
+    multi-table workload, otherwise a strided subset of the process counts.  -> (cells/s, cores, text)."""
+    from oracle import plogp_oracle as po
+    sg = po.SGrid(w.s_list) if w.s_list is not None else po.SGrid(lo=w.s_lo, hi=w.s_hi, step=w.s_step)
+    per_table_cells = w.model_cells() / w.n_tables
+
+    def run_tables(n):
+        t0 = time.perf_counter()
+        for t in range(n):
+            tab = po.Table(w.table_sizes(t), w.gaps[t], w.latency[t])
+            po.select_grid(w.strategy_mask, po.predict_grid(tab, w.strategy_mask, w.P_values(), w.m, sg, w.k_mode))
+        return time.perf_counter() - t0
+
+    def run_stride(stride):
+        P = w.P_values()[::stride]
+        tab = po.Table(w.table_sizes(0), w.gaps[0], w.latency[0])
+        t0 = time.perf_counter()
+        po.select_grid(w.strategy_mask, po.predict_grid(tab, w.strategy_mask, P, w.m, sg, w.k_mode))
+        return time.perf_counter() - t0, per_table_cells * len(P) / w.n_P
+
+    if w.n_tables > 1:
+        t1 = run_tables(1)
+        n = int(max(1, min(w.n_tables, budget_s / max(t1, 1e-6))))
+        dt = run_tables(n)
+        return n * per_table_cells / dt, po.threads(), "first %d of %d tables, full P x m x s grid" % (n, w.n_tables)
+    stride = max(1, w.n_P // 8)
+    dt, cells = run_stride(stride)
+    while dt < budget_s / 4 and stride > 1:
+        stride = max(1, int(stride / min(4.0, budget_s / max(dt, 1e-6))))
+        dt, cells = run_stride(stride)
+    return cells / dt, po.threads(), "every %d-th process count of table 0, all m and s" % stride
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    w = make_workload(args.workload, args.scale, 0)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    rates, text, cores = [], "", 1
+    for i in range(args.warmup + args.steps):
+        r, cores, text = oracle_sample_rate(w, min(20.0, budget))
+        if i >= args.warmup:
+            rates.append(r)
+    value = statistics.mean(rates)
+    print(json.dumps({
+        "impl": "reference", "metric": "model_cells_per_sec", "value": value, "unit": "cells/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.model_cells() / value,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "note": "CPU oracle on a bounded sample; ms_per_step extrapolates to the full step"},
+        "cpu_baseline": {"value": value, "unit": "cells/s", "cores": cores, "kind": "oracle", "sample": text},
+        "e2e": {"value": value, "unit": "cells/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--scale", default="full", choices=["full", "small"], help="small: reduced copy for profiler captures")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import torch.distributed as dist
+    from paper_cs_0408034_b200 import plogp
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = make_workload(args.workload, args.scale, rank)
+    counts = work_counts(w)
+    grid = plogp.GridArgs.from_workload(w)
+    tabs = plogp.Tables.from_workload(w)
+    out = plogp.alloc_decision(w.n_tables, w.n_P, w.n_m)
+    out_bytes = out.strategy.numel() * 13
+    flush = None
+    if out_bytes < (256 << 20):  # outputs do not evict the 126 MB L2 by themselves: write 256 MB between steps
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def step():
+        plogp.select_best(tabs, grid, out=out)
+
+    for _ in range(args.warmup):
+        step()
+        if flush is not None:
+            flush.fill_(1)
+    barrier()
+
+    uuid = str(torch.cuda.get_device_properties(local_rank).uuid)
+    if not uuid.startswith("GPU-"):
+        uuid = "GPU-" + uuid
+    launches0 = plogp.kernel_launches()
+    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    with ClockSampler(uuid) as clocks:
+        barrier()
+        for a, b in events:
+            a.record()
+            step()
+            b.record()
+            if flush is not None:
+                flush.fill_(1)
+        barrier()
+    launches = plogp.kernel_launches() - launches0
+    total_ms = sum(a.elapsed_time(b) for a, b in events)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+
+    # ---- end to end through the public API with host buffers ----
+    e2e_ms, h2d, d2h = None, 0, 0
+    if args.e2e_steps > 0:
+        host = plogp.DecisionTable(*(torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (out.strategy, out.s_bytes, out.time)))
+        h2d = w.sizes.nbytes + w.gaps.nbytes + w.latency.nbytes + w.m.nbytes + (0 if w.s_list is None else w.s_list.nbytes)
+        d2h = sum(t.numel() * t.element_size() for t in (host.strategy, host.s_bytes, host.time))
+
+        def e2e_step():
+            with plogp.Tables.from_workload(w) as tb:   # host arrays -> device (inside plogp_table_load)
+                plogp.select_best(tb, grid, out=out)
+                host.strategy.copy_(out.strategy, non_blocking=True)
+                host.s_bytes.copy_(out.s_bytes, non_blocking=True)
+                host.time.copy_(out.time, non_blocking=True)
+                torch.cuda.synchronize()
+
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        barrier()
+        e2e_ms = (time.perf_counter() - t0) * 1e3 / args.e2e_steps
+        if world > 1:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        del host
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    fma_rate = plogp.fp64_fma_rate(100.0)
+    hbm_gbs, peak_src = measured_peaks()
+    t_alu = counts["fp64_slots"] / fma_rate
+    t_hbm = counts["hbm_bytes"] / (hbm_gbs * 1e9)
+    step_s = ms_per_step * 1e-3
+    alu_bound = t_alu >= t_hbm
+    roofline = {
+        "bound": "alu" if alu_bound else "hbm",
+        "achieved": counts["fp64_slots"] / step_s / 1e12 if alu_bound else counts["hbm_bytes"] / step_s / 1e9,
+        "peak": fma_rate / 1e12 if alu_bound else hbm_gbs,
+        "unit": "T FP64 thread-instr/s" if alu_bound else "GB/s",
+        "frac": max(t_alu, t_hbm) / step_s,
+        "traffic": None,
+        "peak_source": ("DFMA issue rate measured in this run by plogp_fp64_fma_rate (nominal %.2f T/s)" % (NOMINAL_FP64_FMA_RATE / 1e12))
+        if alu_bound else "%s HBM copy bandwidth" % peak_src,
+        "kernel": "sweep_kernel+fused_kernel (step)" if args.workload == "cfg3" else "fused_kernel",
+        "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
+        "hbm_achieved_gbs": counts["hbm_bytes"] / step_s / 1e9, "hbm_peak_gbs": hbm_gbs, "hbm_peak_source": peak_src,
+    }
+
+    line = {
+        "metric": "model_cells_per_sec", "value": world * counts["model_cells"] / step_s, "unit": "cells/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "decision_cells_per_sec": world * counts["decision_cells"] / step_s,
+        "config": {"workload": w.name, "tables_per_gpu": w.n_tables, "P": [w.P_lo, w.P_hi], "n_m": w.n_m,
+                   "n_s": int(len(w.s_values())), "strategy_mask": w.strategy_mask, "model_cells_per_gpu": counts["model_cells"],
+                   "decision_cells_per_gpu": counts["decision_cells"], "parallelism": "tables sharded, %d rank(s)" % world,
+                   "l2": ("outputs (%.1f GB per step) exceed the 126 MB L2" % (out_bytes / 1e9)) if flush is None
+                   else "256 MB written between timed steps to flush L2"},
+        "clocks": clocks.summary(),
+        "e2e": {"value": None if e2e_ms is None else world * counts["model_cells"] / (e2e_ms * 1e-3), "unit": "cells/s",
+                "ms_per_step": e2e_ms, "steps": args.e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "roofline": roofline,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        v, cores, text = oracle_sample_rate(w, 15.0)
+        line["cpu_baseline"] = {"value": v, "unit": "cells/s", "cores": cores, "kind": "oracle", "sample": text}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

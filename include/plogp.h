@@ -135,6 +135,10 @@ const char *plogp_status_string(int status);
 /* Text of the CUDA error behind the calling thread's last PLOGP_E_CUDA ("" if none). */
 const char *plogp_last_cuda_error(void);
 
+/* Number of kernels this library has launched in the calling process so far (all handles, all
+ * threads).  Bookkeeping for benchmarks; no counterpart in the paper. */
+uint64_t plogp_kernel_launches(void);
+
 /*
  * Measurement aid with no counterpart in the paper: runs a register-only chain-free stream of
  * double-precision fused multiply-adds on every SM of the current device for about

@@ -5,6 +5,7 @@
 #include "internal.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <limits>
@@ -17,6 +18,7 @@ using namespace plogp;
 namespace {
 
 thread_local std::string g_cuda_error;
+std::atomic<unsigned long long> g_launches{0};
 
 int cuda_fail(cudaError_t e, const char *what)
 {
@@ -344,6 +346,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             sp.n_pairs = pl.n_pairs; sp.n_ptiles = pl.sweep_ptiles; sp.chunk_len = pl.chunk_len;
             sp.part_time = part_time; sp.part_idx = part_idx; sp.n_seg = pl.n_seg; sp.table0 = t0;
             CK(launch_sweep(sp, nt, st));
+            g_launches += 1;
         }
         if (need_carry) {
             S1Params s{};
@@ -351,6 +354,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             s.n_mtiles = pl.n_mtiles; s.n_ptiles = pl.n_ptiles; s.passes_per_tile = pl.passes_per_tile;
             s.table0 = t0; s.n_tables_launch = nt; s.tile_sum = tile_sum;
             CK(launch_s1_tiles(s, st));
+            g_launches += 2;
         }
         FusedParams fp = out;
         fp.T = h->T; fp.G = pl.G;
@@ -363,6 +367,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
         fp.pair_base = pl.inline_sweep ? nullptr : reinterpret_cast<const int32_t *>(h->d_grid + pl.off_pair_base);
         fp.n_pairs = pl.n_pairs; fp.n_seg = pl.n_seg;
         CK(launch_fused(fp, predict, st));
+        g_launches += 1;
     }
     return PLOGP_OK;
 }
@@ -483,6 +488,8 @@ const char *plogp_status_string(int status)
 
 const char *plogp_last_cuda_error(void) { return g_cuda_error.c_str(); }
 
+uint64_t plogp_kernel_launches(void) { return g_launches.load(); }
+
 double plogp_fp64_fma_rate(double milliseconds)
 {
     if (!(milliseconds > 0.0)) return double(PLOGP_E_INVAL);
@@ -502,6 +509,7 @@ double plogp_fp64_fma_rate(double milliseconds)
         bool ok = true;
         for (int round = 0; round < 3 && ok; ++round) {  // warm-up, calibration, measurement
             ok = cudaEventRecord(e0) == cudaSuccess && launch_fp64_probe(sink, iters, blocks, nullptr) == cudaSuccess &&
+                 (g_launches += 1, true) &&
                  cudaEventRecord(e1) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess &&
                  cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess;
             if (ok && round == 1 && ms > 0.f) iters = int(std::min(2e8, std::max(2000.0, iters * milliseconds / ms)));

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libplogp.so")
 N_STRATEGIES = 13
 SEGMENTED_IDS = (2, 5, 9)
 EXPORTS = ("plogp_table_load", "plogp_table_free", "plogp_predict", "plogp_select_best",
-           "plogp_status_string", "plogp_last_cuda_error", "plogp_fp64_fma_rate")
+           "plogp_status_string", "plogp_last_cuda_error", "plogp_kernel_launches", "plogp_fp64_fma_rate")
 
 OK, E_INVAL, E_NOMEM, E_CUDA, E_RANGE = 0, -1, -2, -3, -4
 
@@ -54,6 +54,8 @@ lib.plogp_status_string.restype = C.c_char_p
 lib.plogp_status_string.argtypes = [C.c_int]
 lib.plogp_last_cuda_error.restype = C.c_char_p
 lib.plogp_last_cuda_error.argtypes = []
+lib.plogp_kernel_launches.restype = C.c_uint64
+lib.plogp_kernel_launches.argtypes = []
 lib.plogp_fp64_fma_rate.restype = C.c_double
 lib.plogp_fp64_fma_rate.argtypes = [C.c_double]
 
@@ -224,3 +226,8 @@ def fp64_fma_rate(milliseconds: float = 50.0) -> float:
     if r < 0:
         raise PlogpError(int(r), "plogp_fp64_fma_rate")
     return r
+
+
+def kernel_launches() -> int:
+    """``plogp_kernel_launches``: kernels launched by the library in this process so far."""
+    return int(lib.plogp_kernel_launches())
