@@ -135,6 +135,38 @@ const char *plogp_status_string(int status);
 /* Text of the CUDA error behind the calling thread's last PLOGP_E_CUDA ("" if none). */
 const char *plogp_last_cuda_error(void);
 
+/*
+ * Scatter Chain predictions without any allocation.  (The paper has no counterpart for this
+ * entry point: it exists for callers that must not allocate device memory while they run, such
+ * as code inside a memory-pool-managed service, a real-time loop, or a section where cudaMalloc's
+ * implicit device synchronisation is not acceptable.)
+ *
+ * Computes the Scatter Chain model, sum_{j=1..P-1} g(j m) + (P-1) L, for one pLogP table, every
+ * P in P_lo..P_hi and every message size in d_m_bytes, exactly as plogp_predict does for strategy
+ * id 11.  The call issues no cudaMalloc, cudaFree or other allocating routine: the partial sums of
+ * its scan live in a fixed 512 KiB array inside the library image, which every device that loads
+ * the library holds until the process exits.
+ *   d_sizes_bytes  DEVICE, [n_bp] strictly increasing sizes (< 2^53); n_bp <= PLOGP_MAX_BREAKPOINTS
+ *   d_gap          DEVICE, [n_bp] finite gaps >= 0
+ *   latency        L, finite, >= 0
+ *   d_m_bytes      DEVICE, [n_m] message sizes; n_m <= PLOGP_STATIC_MAX_M; P_hi * m must stay < 2^53
+ *   d_time         DEVICE, [P_hi - P_lo + 1][n_m] doubles, m fastest; owned by the caller
+ *   stream         cudaStream_t the three kernels are enqueued on; the call does not wait for them
+ * The contents of the device arrays cannot be checked on the host and are trusted.  Sizes beyond
+ * the stated maxima (n_m, P_hi - P_lo + 1 <= PLOGP_STATIC_MAX_P, n_bp) return PLOGP_E_RANGE; other
+ * malformed arguments PLOGP_E_INVAL.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls on a device share the array, which
+ * keeps the previous call's contents; each call overwrites every entry it later reads, so nothing
+ * needs clearing, but two calls whose device work overlaps in time race on it: keep them on one
+ * stream or order them yourself.
+ */
+#define PLOGP_STATIC_MAX_M 256
+#define PLOGP_STATIC_MAX_P 262144
+int plogp_scatter_chain_static(int n_bp, const uint64_t *d_sizes_bytes, const double *d_gap, double latency,
+                               int32_t P_lo, int32_t P_hi, const uint64_t *d_m_bytes, int32_t n_m,
+                               double *d_time, void *stream);
+
 /* Number of kernels this library has launched in the calling process so far (all handles, all
  * threads).  Bookkeeping for benchmarks; no counterpart in the paper. */
 uint64_t plogp_kernel_launches(void);

@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libplogp.so")
 N_STRATEGIES = 13
 SEGMENTED_IDS = (2, 5, 9)
 EXPORTS = ("plogp_table_load", "plogp_table_free", "plogp_predict", "plogp_select_best",
-           "plogp_status_string", "plogp_last_cuda_error", "plogp_kernel_launches", "plogp_fp64_fma_rate")
+           "plogp_status_string", "plogp_last_cuda_error", "plogp_kernel_launches", "plogp_fp64_fma_rate",
+           "plogp_scatter_chain_static")
 
 OK, E_INVAL, E_NOMEM, E_CUDA, E_RANGE = 0, -1, -2, -3, -4
 
@@ -54,6 +55,9 @@ lib.plogp_status_string.restype = C.c_char_p
 lib.plogp_status_string.argtypes = [C.c_int]
 lib.plogp_last_cuda_error.restype = C.c_char_p
 lib.plogp_last_cuda_error.argtypes = []
+lib.plogp_scatter_chain_static.restype = C.c_int
+lib.plogp_scatter_chain_static.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_double, C.c_int32, C.c_int32,
+                                           C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
 lib.plogp_kernel_launches.restype = C.c_uint64
 lib.plogp_kernel_launches.argtypes = []
 lib.plogp_fp64_fma_rate.restype = C.c_double
@@ -231,3 +235,16 @@ def fp64_fma_rate(milliseconds: float = 50.0) -> float:
 def kernel_launches() -> int:
     """``plogp_kernel_launches``: kernels launched by the library in this process so far."""
     return int(lib.plogp_kernel_launches())
+
+
+def scatter_chain_static(d_sizes, d_gap, latency: float, P_lo: int, P_hi: int, d_m, out=None, stream=None):
+    """``plogp_scatter_chain_static``: Scatter Chain times [n_P][n_m] for one table, with every
+    array already on the device (torch int64 sizes / message sizes, float64 gaps).  The library
+    allocates nothing in this call; ``out`` is allocated here, by torch, only when not given."""
+    import torch
+    if out is None:
+        out = torch.empty((P_hi - P_lo + 1, d_m.numel()), dtype=torch.float64, device=d_m.device)
+    _check(lib.plogp_scatter_chain_static(int(d_sizes.numel()), d_sizes.data_ptr(), d_gap.data_ptr(), float(latency),
+                                          int(P_lo), int(P_hi), d_m.data_ptr(), int(d_m.numel()), out.data_ptr(),
+                                          _stream_ptr(stream)), "plogp_scatter_chain_static")
+    return out
