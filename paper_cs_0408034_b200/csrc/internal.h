@@ -80,6 +80,7 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kFusedR = 4;   // process counts per thread and pass in the fused kernel
 constexpr int kSweepR = 8;   // process counts per thread in the sweep kernel
 constexpr int kSweepSub = 256;  // candidates staged per sub-chunk
+constexpr int kSweepU = 4;      // candidates per filter test in the sweep kernel
 constexpr int kMaxInlineS = 64;
 
 size_t fused_smem_bytes(const TableDev &T, const GridDev &G, bool inline_sweep);

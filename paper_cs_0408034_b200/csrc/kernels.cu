@@ -132,11 +132,15 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_kernel(const SweepParams p)
     stage_table(s_tab, p.T, table);
     const double L = p.T.lat[table];
 
+    // A warp owns 256 consecutive process counts (lane + 32 r), so neighbouring cells see similar optima
+    // and the stores below stay coalesced.
+    const int lane = tid & 31, warp = tid >> 5;
+    const int p_first = ptile * (kThreads * R) + warp * (32 * R) + lane;
     double pm1[R], best2[R], best5[R], best9[R], lf[R], lcL[R];
     uint32_t idx2[R], idx5[R], idx9[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        const int pidx = min(ptile * (kThreads * R) + r * kThreads + tid, p.G.n_P - 1);
+        const int pidx = min(p_first + 32 * r, p.G.n_P - 1);
         const int P = P_at(p.G, pidx);
         pm1[r] = static_cast<double>(P - 1);
         lf[r] = static_cast<double>(31 - __clz(P));
@@ -169,31 +173,55 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_kernel(const SweepParams p)
         const double2 *bc = s_bc + buf * kSweepSub;
         const double *qq = s_q + buf * kSweepSub;
         const uint32_t base = static_cast<uint32_t>(s_begin + sub * kSweepSub);
-#pragma unroll 2
-        for (int i = 0; i < kSweepSub; ++i) {
-            const uint32_t sidx = base + i;
-            if (HAS5) {
-                const double2 c = bc[i];
+#pragma unroll 1
+        for (int i = 0; i < kSweepSub; i += kSweepU) {
+            // Hot path: every cell is evaluated (one DFMA); the comparison with the running minimum is
+            // first taken on the high words only, in the integer pipe.  Times are non-negative, so the
+            // high word of a smaller double is never larger: a cell can only improve if that test holds.
+            bool any = false;
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const double t = fma(pm1[r], c.x, c.y);
-                    if (t < best5[r]) { best5[r] = t; idx5[r] = sidx; }
+            for (int u = 0; u < kSweepU; ++u) {
+                if (HAS5) {
+                    const double2 c = bc[i + u];
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+                        any |= __double2hiint(fma(pm1[r], c.x, c.y)) <= __double2hiint(best5[r]);
                 }
-            }
-            if (HAS2 || HAS9) {
-                const double q = qq[i];
-                if (HAS2) {
+                if (HAS2 || HAS9) {
+                    const double q = qq[i + u];
+                    if (HAS2) {
 #pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        const double t = fma(pm1[r], q, L);
-                        if (t < best2[r]) { best2[r] = t; idx2[r] = sidx; }
+                        for (int r = 0; r < R; ++r)
+                            any |= __double2hiint(fma(pm1[r], q, L)) <= __double2hiint(best2[r]);
+                    }
+                    if (HAS9) {
+#pragma unroll
+                        for (int r = 0; r < R; ++r)
+                            any |= __double2hiint(fma(lf[r], q, lcL[r])) <= __double2hiint(best9[r]);
                     }
                 }
-                if (HAS9) {
+            }
+            if (any) {
+                // Exact pass over the same candidates, in ascending order, strict '<' (smallest s on ties).
+#pragma unroll 1
+                for (int u = 0; u < kSweepU; ++u) {
+                    const uint32_t sidx = base + i + u;
+                    const double2 c = bc[i + u];
+                    const double q = qq[i + u];
 #pragma unroll
                     for (int r = 0; r < R; ++r) {
-                        const double t = fma(lf[r], q, lcL[r]);
-                        if (t < best9[r]) { best9[r] = t; idx9[r] = sidx; }
+                        if (HAS5) {
+                            const double t = fma(pm1[r], c.x, c.y);
+                            if (t < best5[r]) { best5[r] = t; idx5[r] = sidx; }
+                        }
+                        if (HAS2) {
+                            const double t = fma(pm1[r], q, L);
+                            if (t < best2[r]) { best2[r] = t; idx2[r] = sidx; }
+                        }
+                        if (HAS9) {
+                            const double t = fma(lf[r], q, lcL[r]);
+                            if (t < best9[r]) { best9[r] = t; idx9[r] = sidx; }
+                        }
                     }
                 }
             }
@@ -207,7 +235,7 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_kernel(const SweepParams p)
         const size_t rbase = (static_cast<size_t>(trel) * p.n_seg + slot) * p.n_pairs + row;
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const int pidx = ptile * (kThreads * R) + r * kThreads + tid;
+            const int pidx = p_first + 32 * r;
             if (pidx < p.G.n_P) {
                 p.part_time[rbase * p.G.n_P + pidx] = best[r];
                 p.part_idx[rbase * p.G.n_P + pidx] = idx[r];
