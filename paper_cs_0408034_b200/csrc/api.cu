@@ -55,6 +55,9 @@ struct Plan {
     bool inline_sweep = true;
     // fused kernel tiling
     int n_mtiles = 0, n_ptiles = 1, passes_per_tile = 1;
+    // decision kernel tiling (short candidate lists)
+    int dec_mgroups = 0, dec_ptiles = 1;
+    size_t carry_bytes_per_table = 0;
     // sweep kernel
     int n_pairs = 0, sweep_ptiles = 0, chunk_len = 0;
     size_t off_pair_m = 0, off_pair_chunk = 0, off_pair_row = 0, off_pair_base = 0;
@@ -222,6 +225,9 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     pl.passes_per_tile = (total_passes + n_ptiles - 1) / n_ptiles;
     pl.n_ptiles = (total_passes + pl.passes_per_tile - 1) / pl.passes_per_tile;
 
+    pl.dec_mgroups = (n_m + kDecMG - 1) / kDecMG;
+    pl.dec_ptiles = (n_P + kDecTileP - 1) / kDecTileP;
+
     // ---- device arrays ----
     std::vector<unsigned char> blob;
     std::vector<uint32_t> m32(n_m);
@@ -286,10 +292,11 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     G.lc_max = std::max(1, ceil_log2(P_hi));
 
     // ---- scratch: sweep partials (per table batch) and Scatter Chain tile prefixes ----
-    const bool need_carry = ((g->strategy_mask >> 11) & 1u) && pl.n_ptiles > 1;
+    const bool s1_on = (g->strategy_mask >> 11) & 1u;
     size_t per_table = 0;
-    if (!pl.inline_sweep) per_table += size_t(pl.n_seg) * pl.n_pairs * n_P * (sizeof(double) + sizeof(uint32_t)) + 64;
-    if (need_carry) per_table += size_t(pl.n_ptiles) * n_m * sizeof(double) + 64;
+    if (!pl.inline_sweep) per_table += size_t(pl.n_seg) * pl.n_pairs * n_P * (sizeof(double) + sizeof(uint32_t)) + 512;
+    if (s1_on && pl.n_ptiles > 1) pl.carry_bytes_per_table = size_t(pl.n_ptiles) * n_m * sizeof(double);
+    per_table += pl.carry_bytes_per_table;
     pl.tables_per_batch = h->T.n_tables;
     if (!pl.inline_sweep && per_table * h->T.n_tables > kSweepScratchLimit)
         pl.tables_per_batch = int(std::max<size_t>(1, kSweepScratchLimit / per_table));
@@ -320,7 +327,12 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
     const Plan &pl = h->plan;
     if (pl.empty) return PLOGP_OK;
     const bool s1 = (pl.G.mask >> 11) & 1u;
-    const bool need_carry = s1 && pl.n_ptiles > 1;
+    // Short candidate lists with segmented strategies: the lane<->P decision kernel; everything else
+    // (predictions, long lists reduced by the sweep kernel, Scatter-only grids) goes through fused_kernel.
+    const bool use_decide = !predict && pl.inline_sweep && pl.n_seg > 0;
+    const int n_ptiles = pl.n_ptiles;
+    const int passes_per_tile = pl.passes_per_tile;
+    const bool need_carry = s1 && n_ptiles > 1;
 
     for (int t0 = 0; t0 < h->T.n_tables; t0 += pl.tables_per_batch) {
         const int nt = std::min(pl.tables_per_batch, h->T.n_tables - t0);
@@ -351,13 +363,28 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
         if (need_carry) {
             S1Params s{};
             s.T = h->T; s.G = pl.G;
-            s.n_mtiles = pl.n_mtiles; s.n_ptiles = pl.n_ptiles; s.passes_per_tile = pl.passes_per_tile;
+            s.n_mtiles = pl.n_mtiles; s.n_ptiles = n_ptiles; s.passes_per_tile = passes_per_tile;
             s.table0 = t0; s.n_tables_launch = nt; s.tile_sum = tile_sum;
             CK(launch_s1_tiles(s, st));
             g_launches += 2;
         }
+        GridDev Gf = pl.G;
+        if (use_decide) {
+            // Broadcast half with lanes <-> P; the Scatter half (no candidate lists) follows in fused_kernel.
+            DecideParams dp{};
+            dp.T = h->T; dp.G = pl.G;
+            dp.G.mask &= 0x3FFu;
+            dp.n_mgroups = pl.dec_mgroups; dp.n_ptiles = pl.dec_ptiles;
+            dp.table0 = t0; dp.n_tables_launch = nt;
+            dp.d_strategy = out.d_strategy; dp.d_sbytes = out.d_sbytes; dp.d_time = out.d_time;
+            CK(launch_decide(dp, st));
+            g_launches += 1;
+            Gf.mask &= 0x1C00u;
+            Gf.n_s = 0;
+            if (!Gf.mask) continue;
+        }
         FusedParams fp = out;
-        fp.T = h->T; fp.G = pl.G;
+        fp.T = h->T; fp.G = Gf;
         fp.n_mtiles = pl.n_mtiles; fp.n_ptiles = pl.n_ptiles; fp.passes_per_tile = pl.passes_per_tile;
         fp.table0 = t0; fp.n_tables_launch = nt;
         fp.s1_carry = tile_sum;
@@ -383,7 +410,7 @@ int plogp_table_load(int n_tables, int n_bp, const uint64_t *sizes_bytes, int si
     if (n_tables < 1 || n_bp < 2) return PLOGP_E_INVAL;
     if (n_bp > PLOGP_MAX_BREAKPOINTS) return PLOGP_E_RANGE;
     int npad = 2;
-    while (npad < n_bp - 1) npad <<= 1;
+    while (npad < n_bp) npad <<= 1;  // >= n_bp: at least one +inf key follows the last interval
 
     std::vector<double> tab, lat;
     try {

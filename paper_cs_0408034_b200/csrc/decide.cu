@@ -1,0 +1,296 @@
+// decide_kernel: Broadcast half of the decision table (Sections 1 and 5 of the paper) for short
+// candidate lists, with lanes mapped to the process count P.  (The Scatter half has no candidate
+// lists and goes through fused_kernel.)
+//
+// One CTA owns one table, a group of 8 message sizes and a tile of 512 process counts (4 warps x
+// 32 lanes x 4 cells).  For a fixed (m, s) the segmented models of Table 1 are lines in P, so the
+// CTA computes the line coefficients once per (m, s) into shared memory and every lane reads them
+// with one broadcast load.  Each model cell is evaluated with one DFMA.  The comparison with the
+// running minimum is first made on the high 32 bits in the integer pipe (times are non-negative,
+// so a smaller double never has a larger high word); only chunks of candidates in which some cell
+// can improve run the exact FP64 compare-and-select pass.  To make that pass rare, each warp first
+// finds the best candidate for the process count in the middle of its range (one candidate per
+// lane, shuffle argmin) and evaluates that candidate's chunk first: neighbouring process counts
+// nearly always share the optimum, and for ids 2 and 9 the optimum does not depend on P at all.
+//
+// Results are staged in shared memory as [m][P] and written out as rows of 8 consecutive m.
+#include "device_common.cuh"
+
+#include <algorithm>
+
+namespace plogp {
+
+namespace {
+
+constexpr int kDecStride = kDecTileP + 2;  // doubles per staged row: keeps the transposed reads conflict-free
+
+struct DecSmem {
+    double *tab, *gs, *cQ, *gm, *st_time;
+    double2 *cBC;
+    uint8_t *st_id, *st_si;
+};
+
+__host__ __device__ inline size_t dec_layout(int npad, int nsp, unsigned char *base, DecSmem *o)
+{
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off += (bytes + 15) & ~size_t(15); return at; };
+    const size_t o_tab = take(3 * size_t(npad) * 8), o_gs = take(size_t(nsp) * 8), o_BC = take(size_t(nsp) * 16),
+                 o_Q = take(size_t(nsp) * 8), o_gm = take(kDecMG * 8), o_t = take(size_t(kDecMG) * kDecStride * 8),
+                 o_id = take(size_t(kDecMG) * (kDecTileP + 16)), o_si = take(size_t(kDecMG) * (kDecTileP + 16));
+    if (o) {
+        o->tab = reinterpret_cast<double *>(base + o_tab); o->gs = reinterpret_cast<double *>(base + o_gs);
+        o->cBC = reinterpret_cast<double2 *>(base + o_BC); o->cQ = reinterpret_cast<double *>(base + o_Q);
+        o->gm = reinterpret_cast<double *>(base + o_gm); o->st_time = reinterpret_cast<double *>(base + o_t);
+        o->st_id = base + o_id; o->st_si = base + o_si;
+    }
+    return off;
+}
+
+constexpr uint8_t kSiNone = 255;      // winner is an unsegmented strategy
+constexpr uint8_t kSiWhole = 254;     // segmented winner with no fitting candidate: the whole message
+
+
+}  // namespace
+
+__global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecideParams p)
+{
+    constexpr int R = kDecR, U = kDecU;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int npad = p.T.npad;
+    const int nsp = (max(p.G.n_s, 1) + U - 1) / U * U;
+    DecSmem sm;
+    dec_layout(npad, nsp, smem_raw, &sm);
+    const uint32_t mask = p.G.mask;
+
+    int b = blockIdx.x;
+    const int mgroup = b % p.n_mgroups;
+    b /= p.n_mgroups;
+    const int ptile = b % p.n_ptiles;
+    const int trel = b / p.n_ptiles;
+    const int table = p.table0 + trel;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int m0 = mgroup * kDecMG;
+    const int n_mi = min(kDecMG, p.G.n_m - m0);
+
+    stage_table(sm.tab, p.T, table);
+    __syncthreads();
+    const double L = p.T.lat[table];
+    for (int si = tid; si < p.G.n_s; si += kDecThreads)
+        sm.gs[si] = gap_at(sm.tab, npad, static_cast<double>(s_at(p.G, si)));
+    if (tid >= kDecThreads - kDecMG) {  // g(m) of the group's message sizes, by the last threads
+        const int mi = tid - (kDecThreads - kDecMG);
+        if (mi < n_mi) sm.gm[mi] = gap_at(sm.tab, npad, static_cast<double>(p.G.m_list[m0 + mi]));
+    }
+    const double g1 = gap_at(sm.tab, npad, 1.0);
+    const double rdv = 2.0 * g1 + 3.0 * L;  // rendezvous handshake: 2 g(1) + 3 L
+
+    // this thread's cells: process counts at tile offset warp*128 + r*32 + lane
+    const int p_first = ptile * kDecTileP + warp * (32 * R) + lane;
+    int Pv[R];
+    double pm1[R], lf[R], lc[R], lcL[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int pidx = p_first + 32 * r;
+        Pv[r] = P_at(p.G, min(pidx, p.G.n_P - 1));
+        pm1[r] = static_cast<double>(Pv[r] - 1);
+        lf[r] = static_cast<double>(31 - __clz(Pv[r]));
+        lc[r] = static_cast<double>(32 - __clz(Pv[r] - 1));
+        lcL[r] = lc[r] * L;
+    }
+    // the warp's pilot process count (middle of its range, clamped to the grid)
+    const int P_mid = P_at(p.G, min(ptile * kDecTileP + warp * (32 * R) + 16 * R, p.G.n_P - 1));
+    const double pm1_mid = static_cast<double>(P_mid - 1);
+
+    const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
+
+    // transposed write-out of the staged group: rows of n_mi consecutive m per process count
+    auto write_out = [&](int coll) {
+        const int mi = lane & 7, prow = lane >> 3;
+        if (mi < n_mi) {
+            const uint32_t m_u = p.G.m_list[m0 + mi];
+            for (int pr = warp * 4 + prow; pr < kDecTileP; pr += kDecWarps * 4) {
+                const int pidx = ptile * kDecTileP + pr;
+                if (pidx >= p.G.n_P) break;
+                const size_t o = (static_cast<size_t>(table) * 2 + coll) * plane + static_cast<size_t>(pidx) * p.G.n_m + m0 + mi;
+                const uint8_t si = sm.st_si[mi * (kDecTileP + 16) + pr];
+                p.d_time[o] = sm.st_time[mi * kDecStride + pr];
+                p.d_strategy[o] = sm.st_id[mi * (kDecTileP + 16) + pr];
+                p.d_sbytes[o] = si == kSiNone ? 0u : (si == kSiWhole ? m_u : s_at(p.G, si));
+            }
+        }
+    };
+
+    // =============================== Broadcast (Table 1) ===============================
+    if (mask & 0x3FFu) {
+        for (int mi = 0; mi < n_mi; ++mi) {
+            const int midx = m0 + mi;
+            const uint32_t m_u = p.G.m_list[midx];
+            const int ns = p.G.ns_of_m[midx];
+            const int nsv = max(ns, 1);                 // candidates actually evaluated
+            const int n_chunks = (nsv + U - 1) / U;
+
+            __syncthreads();  // the previous message size is done with the coefficient arrays
+            const double gm = sm.gm[mi];
+            // line coefficients per candidate (Section 2's k, Table 1's segmented rows)
+            for (int si = tid; si < n_chunks * U; si += kDecThreads) {
+                double B = CUDART_INF, C = CUDART_INF, Q = CUDART_INF;  // padding never wins
+                if (si < ns) {
+                    const double gs = sm.gs[si];
+                    const double k = static_cast<double>(segments(m_u, s_at(p.G, si), p.G.k_mode));
+                    B = gs + L; C = gs * (k - 1.0); Q = gs * k;
+                } else if (ns == 0 && si == 0) {        // nothing fits: the whole message, k = 1
+                    B = gm + L; C = 0.0; Q = gm;
+                }
+                sm.cBC[si] = make_double2(B, C); sm.cQ[si] = Q;
+            }
+            __syncthreads();
+
+            double bt[R];
+            int bid[R];
+            uint32_t bsi[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) { bt[r] = CUDART_INF; bid[r] = 255; bsi[r] = kSiNone; }
+            auto consider = [&](int id, const double *val, const uint32_t *sval) {
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+                    if (val[r] < bt[r]) { bt[r] = val[r]; bid[r] = id; bsi[r] = sval ? sval[r] : kSiNone; }
+            };
+
+            // Pilot: the candidate that is best for the process count in the middle of the warp's range.
+            // Only a guess that orders the work (float precision, index in the low bits of the key).
+            auto pilot_chunk = [&](auto eval_mid) {
+                unsigned key = 0xFFFFFFFFu;
+                for (int c0 = 0; c0 < nsv; c0 += 32) {
+                    const int cand = c0 + lane;
+                    if (cand < nsv) {
+                        const unsigned k = (__float_as_uint(static_cast<float>(eval_mid(cand))) & ~63u) | static_cast<unsigned>(cand);
+                        key = min(key, k);
+                    }
+                }
+                return static_cast<int>(__reduce_min_sync(0xffffffffu, key) & 63u) / U;
+            };
+            // Segmented model reduced over the candidates: eval(r, cand) is the model cell.
+            auto segmented = [&](int id, int cp, auto eval) {
+                double st[R];
+                uint32_t si[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) { st[r] = CUDART_INF; si[r] = 0; }
+                // the pilot's chunk first, ascending, strict '<'
+#pragma unroll 1
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t cand = cp * U + u;
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const double t = eval(r, cand);
+                        if (t < st[r]) { st[r] = t; si[r] = cand; }
+                    }
+                }
+                for (int chunk = 0; chunk < n_chunks; ++chunk) {
+                    if (chunk == cp) continue;
+                    bool any = false;
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+#pragma unroll
+                        for (int r = 0; r < R; ++r)
+                            any |= __double2hiint(eval(r, chunk * U + u)) <= __double2hiint(st[r]);
+                    }
+                    if (any) {  // exact pass; candidates arrive out of order, so ties go to the smaller index
+#pragma unroll 1
+                        for (int u = 0; u < U; ++u) {
+                            const uint32_t cand = chunk * U + u;
+#pragma unroll
+                            for (int r = 0; r < R; ++r) {
+                                const double t = eval(r, cand);
+                                if (t < st[r] || (t == st[r] && cand < si[r])) { st[r] = t; si[r] = cand; }
+                            }
+                        }
+                    }
+                }
+                if (ns == 0) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) si[r] = kSiWhole;
+                }
+                consider(id, st, si);
+            };
+            // ids 2 and 9 are a_P * Q(s) + c_P with a_P > 0: their best candidate is the same for every P
+            int cpQ = 0;
+            if (mask & ((1u << 2) | (1u << 9))) cpQ = pilot_chunk([&](int cand) { return sm.cQ[cand]; });
+
+            double v[R];
+            if (mask & 1u) {  // Flat Tree
+#pragma unroll
+                for (int r = 0; r < R; ++r) v[r] = fma(pm1[r], gm, L);
+                consider(0, v, nullptr);
+            }
+            if ((mask >> 1) & 1u) {  // Flat Tree Rendezvous
+#pragma unroll
+                for (int r = 0; r < R; ++r) v[r] = fma(pm1[r], gm, rdv);
+                consider(1, v, nullptr);
+            }
+            if ((mask >> 2) & 1u)  // Segmented Flat Tree
+                segmented(2, cpQ, [&](int r, int cand) { return fma(pm1[r], sm.cQ[cand], L); });
+            if ((mask >> 3) & 1u) {  // Chain
+#pragma unroll
+                for (int r = 0; r < R; ++r) v[r] = pm1[r] * (gm + L);
+                consider(3, v, nullptr);
+            }
+            if ((mask >> 4) & 1u) {  // Chain Rendezvous
+#pragma unroll
+                for (int r = 0; r < R; ++r) v[r] = pm1[r] * (gm + rdv);
+                consider(4, v, nullptr);
+            }
+            if ((mask >> 5) & 1u) {  // Segmented Chain
+                const int cp5 = pilot_chunk([&](int cand) { const double2 c = sm.cBC[cand]; return fma(pm1_mid, c.x, c.y); });
+                segmented(5, cp5, [&](int r, int cand) { const double2 c = sm.cBC[cand]; return fma(pm1[r], c.x, c.y); });
+            }
+            if ((mask >> 6) & 1u) {  // Binary Tree (the printed bound)
+#pragma unroll
+                for (int r = 0; r < R; ++r) v[r] = lc[r] * fma(2.0, gm, L);
+                consider(6, v, nullptr);
+            }
+            if ((mask >> 7) & 1u) {  // Binomial Tree
+#pragma unroll
+                for (int r = 0; r < R; ++r) v[r] = fma(lf[r], gm, lcL[r]);
+                consider(7, v, nullptr);
+            }
+            if ((mask >> 8) & 1u) {  // Binomial Tree Rendezvous
+#pragma unroll
+                for (int r = 0; r < R; ++r) v[r] = fma(lf[r], gm, lc[r] * rdv);
+                consider(8, v, nullptr);
+            }
+            if ((mask >> 9) & 1u)  // Segmented Binomial Tree
+                segmented(9, cpQ, [&](int r, int cand) { return fma(lf[r], sm.cQ[cand], lcL[r]); });
+
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int pr = warp * (32 * R) + 32 * r + lane;
+                sm.st_time[mi * kDecStride + pr] = bt[r];
+                sm.st_id[mi * (kDecTileP + 16) + pr] = static_cast<uint8_t>(bid[r]);
+                sm.st_si[mi * (kDecTileP + 16) + pr] = static_cast<uint8_t>(bsi[r]);
+            }
+        }
+        __syncthreads();
+        write_out(0);
+    }
+}
+
+size_t decide_smem_bytes(const TableDev &T, const GridDev &G)
+{
+    const int nsp = (std::max(G.n_s, 1) + kDecU - 1) / kDecU * kDecU;
+    return dec_layout(T.npad, nsp, nullptr, nullptr);
+}
+
+cudaError_t launch_decide(const DecideParams &p, cudaStream_t st)
+{
+    const size_t smem = decide_smem_bytes(p.T, p.G);
+    cudaError_t e = cudaSuccess;
+    if (smem > 48 * 1024)
+        e = cudaFuncSetAttribute(decide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    const long long blocks = static_cast<long long>(p.n_mgroups) * p.n_ptiles * p.n_tables_launch;
+    if (blocks <= 0 || blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    decide_kernel<<<static_cast<unsigned>(blocks), kDecThreads, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace plogp

@@ -1,0 +1,112 @@
+// Device helpers shared by the kernels: table staging into shared memory, g(x), grid accessors.
+#pragma once
+
+#include "internal.h"
+
+#include <math_constants.h>
+
+namespace plogp {
+
+// ------------------------------------------------------------------------------------------
+// Table staging and g(x)
+// ------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
+{
+    unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src));
+}
+
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.commit_group;\n" ::: "memory");
+    asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+}
+
+// Copies one table (key | gap | slope, 3*npad doubles) into shared memory with 16-byte
+// asynchronous copies.  The caller synchronises the CTA afterwards.
+__device__ __forceinline__ void stage_table(double *s_tab, const TableDev &T, int table)
+{
+    const double *src = T.tab + static_cast<size_t>(table) * 3 * T.npad;
+    const int n16 = (3 * T.npad) >> 1;
+    for (int i = threadIdx.x; i < n16; i += blockDim.x) cp_async16(s_tab + 2 * i, src + 2 * i);
+    cp_async_wait_all();
+}
+
+// g(x) of Section 2 on the staged table: branch-free search of the interval that starts at or
+// below x (keys beyond the last interval are +inf), then one fused multiply-add along that
+// interval's line.  x below the first size is held at the first gap (dx clamped to 0); x above
+// the last size continues the last interval's line.
+__device__ __forceinline__ double gap_at(const double *s_tab, int npad, double x)
+{
+    int i = 0;
+#pragma unroll 1
+    for (int step = npad >> 1; step > 0; step >>= 1) {
+        const int j = i + step;
+        i = (s_tab[j] <= x) ? j : i;
+    }
+    const double dx = fmax(x - s_tab[i], 0.0);
+    return fma(dx, s_tab[2 * npad + i], s_tab[npad + i]);
+}
+
+__device__ __forceinline__ int P_at(const GridDev &G, int pidx)
+{
+    return G.P_list ? G.P_list[pidx] : G.P_lo + pidx;
+}
+
+__device__ __forceinline__ uint32_t s_at(const GridDev &G, int si)
+{
+    return G.s_list ? G.s_list[si] : G.s_lo + static_cast<uint32_t>(si) * G.s_step;
+}
+
+// k of Section 2: number of segments of size s in a message of m bytes.
+__device__ __forceinline__ uint32_t segments(uint32_t m, uint32_t s, int k_mode)
+{
+    const uint32_t q = m / s;
+    return q + ((k_mode == 0 && q * s != m) ? 1u : 0u);
+}
+
+// Interval search alone: largest i with key[i] <= x (0 when x is below the table).
+__device__ __forceinline__ int interval_of(const double *s_tab, int npad, double x)
+{
+    int i = 0;
+#pragma unroll 1
+    for (int step = npad >> 1; step > 0; step >>= 1) {
+        const int j = i + step;
+        i = (s_tab[j] <= x) ? j : i;
+    }
+    return i;
+}
+
+// g(x) for a caller that walks x upwards: `i` is the interval of the previous, smaller argument and
+// is advanced to the interval of x (keys past the last interval are +inf, and npad >= n_bp leaves
+// at least one such key, so the walk stops inside the array).
+__device__ __forceinline__ double gap_walk(const double *s_tab, int npad, double x, int &i)
+{
+    while (s_tab[i + 1] <= x) ++i;
+    const double dx = fmax(x - s_tab[i], 0.0);
+    return fma(dx, s_tab[2 * npad + i], s_tab[npad + i]);
+}
+
+// One term of the Scatter Chain sum for the process count at index pidx: the gaps g(j m) for j
+// from the previous listed process count (1 before the first) up to P-1.  For a contiguous
+// range of P this is the single gap g((P-1) m); longer runs are added with compensation.
+// `i` carries the table interval from one call to the next (arguments must not decrease); pass
+// a negative value on the first call.
+__device__ __forceinline__ double s1_term(const double *s_tab, int npad, const GridDev &G, int pidx, double md, int &i)
+{
+    const int jhi = P_at(G, pidx) - 1;
+    const int jlo = pidx == 0 ? 1 : P_at(G, pidx - 1);
+    if (i < 0) i = interval_of(s_tab, npad, static_cast<double>(jlo) * md);
+    if (jlo == jhi) return gap_walk(s_tab, npad, static_cast<double>(jlo) * md, i);
+    double sum = 0.0, comp = 0.0;
+    for (int j = jlo; j <= jhi; ++j) {
+        const double y = gap_walk(s_tab, npad, static_cast<double>(j) * md, i) - comp;
+        const double t = sum + y;
+        comp = (t - sum) - y;
+        sum = t;
+    }
+    return sum;
+}
+
+}  // namespace plogp

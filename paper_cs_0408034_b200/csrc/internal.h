@@ -11,7 +11,8 @@ namespace plogp {
 //   key[npad]   breakpoint sizes usable as interval starts (index <= n_bp-2), +inf beyond
 //   gap[npad]   g at the interval start
 //   slope[npad] (g[i+1]-g[i]) / (size[i+1]-size[i])
-// npad is a power of two >= n_bp-1, so the interval search needs no bounds checks.
+// npad is a power of two >= n_bp, so the interval search needs no bounds checks and an upward
+// walk always meets a +inf key.
 struct TableDev {
     const double *tab;  // [n_tables][3*npad]
     const double *lat;  // [n_tables]
@@ -75,6 +76,24 @@ struct S1Params {
     double *tile_sum;  // [n_tables_launch][n_ptiles][n_m]
 };
 
+// Decision kernel for short candidate lists (lanes <-> P): see decide.cu
+struct DecideParams {
+    TableDev T;
+    GridDev G;
+    int n_mgroups, n_ptiles;
+    int table0, n_tables_launch;
+    uint8_t *d_strategy;
+    uint32_t *d_sbytes;
+    double *d_time;
+};
+
+constexpr int kDecThreads = 128;
+constexpr int kDecWarps = kDecThreads / 32;
+constexpr int kDecR = 4;                               // process counts per thread
+constexpr int kDecTileP = kDecThreads * kDecR;         // 512 process counts per CTA
+constexpr int kDecMG = 8;                              // message sizes per CTA
+constexpr int kDecU = 4;                               // candidates per filter test
+
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kFusedR = 4;   // process counts per thread and pass in the fused kernel
@@ -87,6 +106,8 @@ size_t fused_smem_bytes(const TableDev &T, const GridDev &G, bool inline_sweep);
 cudaError_t launch_fused(const FusedParams &p, bool predict, cudaStream_t st);
 cudaError_t launch_sweep(const SweepParams &p, int n_tables_launch, cudaStream_t st);
 cudaError_t launch_s1_tiles(const S1Params &p, cudaStream_t st);
+size_t decide_smem_bytes(const TableDev &T, const GridDev &G);
+cudaError_t launch_decide(const DecideParams &p, cudaStream_t st);
 cudaError_t launch_fp64_probe(double *d_sink, int iters, int blocks, cudaStream_t st);
 
 }  // namespace plogp

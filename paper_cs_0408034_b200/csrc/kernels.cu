@@ -11,88 +11,9 @@
 //                  written as full, aligned segments).  Evaluates all enabled strategies, runs short
 //                  candidate lists inline, block-scans the Scatter Chain sum over P, and writes
 //                  either the predicted planes or the decision table.
-#include "internal.h"
-
-#include <math_constants.h>
+#include "device_common.cuh"
 
 namespace plogp {
-
-// ------------------------------------------------------------------------------------------
-// Table staging and g(x)
-// ------------------------------------------------------------------------------------------
-
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
-{
-    unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src));
-}
-
-__device__ __forceinline__ void cp_async_wait_all()
-{
-    asm volatile("cp.async.commit_group;\n" ::: "memory");
-    asm volatile("cp.async.wait_group 0;\n" ::: "memory");
-}
-
-// Copies one table (key | gap | slope, 3*npad doubles) into shared memory with 16-byte
-// asynchronous copies.  The caller synchronises the CTA afterwards.
-__device__ __forceinline__ void stage_table(double *s_tab, const TableDev &T, int table)
-{
-    const double *src = T.tab + static_cast<size_t>(table) * 3 * T.npad;
-    const int n16 = (3 * T.npad) >> 1;
-    for (int i = threadIdx.x; i < n16; i += blockDim.x) cp_async16(s_tab + 2 * i, src + 2 * i);
-    cp_async_wait_all();
-}
-
-// g(x) of Section 2 on the staged table: branch-free search of the interval that starts at or
-// below x (keys beyond the last interval are +inf), then one fused multiply-add along that
-// interval's line.  x below the first size is held at the first gap (dx clamped to 0); x above
-// the last size continues the last interval's line.
-__device__ __forceinline__ double gap_at(const double *s_tab, int npad, double x)
-{
-    int i = 0;
-#pragma unroll 1
-    for (int step = npad >> 1; step > 0; step >>= 1) {
-        const int j = i + step;
-        i = (s_tab[j] <= x) ? j : i;
-    }
-    const double dx = fmax(x - s_tab[i], 0.0);
-    return fma(dx, s_tab[2 * npad + i], s_tab[npad + i]);
-}
-
-__device__ __forceinline__ int P_at(const GridDev &G, int pidx)
-{
-    return G.P_list ? G.P_list[pidx] : G.P_lo + pidx;
-}
-
-__device__ __forceinline__ uint32_t s_at(const GridDev &G, int si)
-{
-    return G.s_list ? G.s_list[si] : G.s_lo + static_cast<uint32_t>(si) * G.s_step;
-}
-
-// k of Section 2: number of segments of size s in a message of m bytes.
-__device__ __forceinline__ uint32_t segments(uint32_t m, uint32_t s, int k_mode)
-{
-    const uint32_t q = m / s;
-    return q + ((k_mode == 0 && q * s != m) ? 1u : 0u);
-}
-
-// One term of the Scatter Chain sum for the process count at index pidx: the gaps g(j m) for j
-// from the previous listed process count (1 before the first) up to P-1.  For a contiguous
-// range of P this is the single gap g((P-1) m); longer runs are added with compensation.
-__device__ __forceinline__ double s1_term(const double *s_tab, int npad, const GridDev &G, int pidx, double md)
-{
-    const int jhi = P_at(G, pidx) - 1;
-    const int jlo = pidx == 0 ? 1 : P_at(G, pidx - 1);
-    if (jlo == jhi) return gap_at(s_tab, npad, static_cast<double>(jlo) * md);
-    double sum = 0.0, comp = 0.0;
-    for (int j = jlo; j <= jhi; ++j) {
-        const double y = gap_at(s_tab, npad, static_cast<double>(j) * md) - comp;
-        const double t = sum + y;
-        comp = (t - sum) - y;
-        sum = t;
-    }
-    return sum;
-}
 
 // ------------------------------------------------------------------------------------------
 // Segment sweep: partial minima over one chunk of candidates (Section 3.1 search)
@@ -178,50 +99,60 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_kernel(const SweepParams p)
             // Hot path: every cell is evaluated (one DFMA); the comparison with the running minimum is
             // first taken on the high words only, in the integer pipe.  Times are non-negative, so the
             // high word of a smaller double is never larger: a cell can only improve if that test holds.
-            bool any = false;
+            bool any5 = false, any2 = false, any9 = false;
 #pragma unroll
             for (int u = 0; u < kSweepU; ++u) {
                 if (HAS5) {
                     const double2 c = bc[i + u];
 #pragma unroll
                     for (int r = 0; r < R; ++r)
-                        any |= __double2hiint(fma(pm1[r], c.x, c.y)) <= __double2hiint(best5[r]);
+                        any5 |= __double2hiint(fma(pm1[r], c.x, c.y)) <= __double2hiint(best5[r]);
                 }
                 if (HAS2 || HAS9) {
                     const double q = qq[i + u];
                     if (HAS2) {
 #pragma unroll
                         for (int r = 0; r < R; ++r)
-                            any |= __double2hiint(fma(pm1[r], q, L)) <= __double2hiint(best2[r]);
+                            any2 |= __double2hiint(fma(pm1[r], q, L)) <= __double2hiint(best2[r]);
                     }
                     if (HAS9) {
 #pragma unroll
                         for (int r = 0; r < R; ++r)
-                            any |= __double2hiint(fma(lf[r], q, lcL[r])) <= __double2hiint(best9[r]);
+                            any9 |= __double2hiint(fma(lf[r], q, lcL[r])) <= __double2hiint(best9[r]);
                     }
                 }
             }
-            if (any) {
-                // Exact pass over the same candidates, in ascending order, strict '<' (smallest s on ties).
+            // Exact passes over the same candidates, in ascending order, strict '<' (smallest s on ties).
+            if (HAS5 && any5) {
 #pragma unroll 1
                 for (int u = 0; u < kSweepU; ++u) {
-                    const uint32_t sidx = base + i + u;
                     const double2 c = bc[i + u];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const double t = fma(pm1[r], c.x, c.y);
+                        if (t < best5[r]) { best5[r] = t; idx5[r] = base + i + u; }
+                    }
+                }
+            }
+            if (HAS2 && any2) {
+#pragma unroll 1
+                for (int u = 0; u < kSweepU; ++u) {
                     const double q = qq[i + u];
 #pragma unroll
                     for (int r = 0; r < R; ++r) {
-                        if (HAS5) {
-                            const double t = fma(pm1[r], c.x, c.y);
-                            if (t < best5[r]) { best5[r] = t; idx5[r] = sidx; }
-                        }
-                        if (HAS2) {
-                            const double t = fma(pm1[r], q, L);
-                            if (t < best2[r]) { best2[r] = t; idx2[r] = sidx; }
-                        }
-                        if (HAS9) {
-                            const double t = fma(lf[r], q, lcL[r]);
-                            if (t < best9[r]) { best9[r] = t; idx9[r] = sidx; }
-                        }
+                        const double t = fma(pm1[r], q, L);
+                        if (t < best2[r]) { best2[r] = t; idx2[r] = base + i + u; }
+                    }
+                }
+            }
+            if (HAS9 && any9) {
+#pragma unroll 1
+                for (int u = 0; u < kSweepU; ++u) {
+                    const double q = qq[i + u];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const double t = fma(lf[r], q, lcL[r]);
+                        if (t < best9[r]) { best9[r] = t; idx9[r] = base + i + u; }
                     }
                 }
             }
@@ -272,11 +203,12 @@ __global__ void __launch_bounds__(kThreads) s1_tile_sum_kernel(const S1Params p)
     __syncthreads();
 
     double acc = 0.0;
+    int walk = -1;
     for (int pass = 0; pass < p.passes_per_tile; ++pass) {
         const int p0 = (ptile * p.passes_per_tile + pass) * (kWarps * R) + warp * R;
 #pragma unroll
         for (int r = 0; r < R; ++r)
-            if (p0 + r < p.G.n_P) acc += s1_term(s_tab, p.T.npad, p.G, p0 + r, md);
+            if (p0 + r < p.G.n_P) acc += s1_term(s_tab, p.T.npad, p.G, p0 + r, md, walk);
     }
     s_red[warp * 32 + lane] = acc;
     __syncthreads();
@@ -394,6 +326,7 @@ __global__ void __launch_bounds__(kThreads) fused_kernel(const FusedParams p)
     __syncthreads();
 
     double carry = 0.0;
+    int s1_walk = -1;  // table interval of this thread's last Scatter Chain argument
     if (p.s1_carry) carry = p.s1_carry[(static_cast<size_t>(trel) * p.n_ptiles + ptile) * p.G.n_m + midx_c];
 
     const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
@@ -419,7 +352,7 @@ __global__ void __launch_bounds__(kThreads) fused_kernel(const FusedParams p)
             double run = 0.0;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                if (ok[r]) run += s1_term(sm.tab, npad, p.G, p0 + r, md);
+                if (ok[r]) run += s1_term(sm.tab, npad, p.G, p0 + r, md, s1_walk);
                 s1sum[r] = run;
             }
             double *tot = sm.tot + (pass & 1) * (kWarps * 32);
