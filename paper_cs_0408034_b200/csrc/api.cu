@@ -393,7 +393,8 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
         fp.part_idx = part_idx;
         fp.pair_base = pl.inline_sweep ? nullptr : reinterpret_cast<const int32_t *>(h->d_grid + pl.off_pair_base);
         fp.n_pairs = pl.n_pairs; fp.n_seg = pl.n_seg;
-        CK(launch_fused(fp, predict, st));
+        if (!predict && (Gf.mask & 0x3FFu) == 0) CK(launch_scatter(fp, st));
+        else CK(launch_fused(fp, predict, st));
         g_launches += 1;
     }
     return PLOGP_OK;

@@ -78,30 +78,47 @@ __device__ __forceinline__ int interval_of(const double *s_tab, int npad, double
     return i;
 }
 
-// g(x) for a caller that walks x upwards: `i` is the interval of the previous, smaller argument and
-// is advanced to the interval of x (keys past the last interval are +inf, and npad >= n_bp leaves
-// at least one such key, so the walk stops inside the array).
-__device__ __forceinline__ double gap_walk(const double *s_tab, int npad, double x, int &i)
-{
-    while (s_tab[i + 1] <= x) ++i;
-    const double dx = fmax(x - s_tab[i], 0.0);
-    return fma(dx, s_tab[2 * npad + i], s_tab[npad + i]);
-}
+// g(x) for a caller whose arguments never decrease: the current interval's line is kept in
+// registers and shared memory is touched only when x crosses into the next interval (keys past
+// the last interval are +inf, and npad >= n_bp leaves at least one such key, so the walk stops
+// inside the array).
+struct GapWalk {
+    int i = -1;
+    double key, next, slope, gap;
+
+    __device__ __forceinline__ void load(const double *s_tab, int npad)
+    {
+        key = s_tab[i];
+        next = s_tab[i + 1];
+        slope = s_tab[2 * npad + i];
+        gap = s_tab[npad + i];
+    }
+    __device__ __forceinline__ double at(const double *s_tab, int npad, double x)
+    {
+        if (i < 0) {
+            i = interval_of(s_tab, npad, x);
+            load(s_tab, npad);
+        }
+        while (x >= next) {
+            ++i;
+            load(s_tab, npad);
+        }
+        return fma(fmax(x - key, 0.0), slope, gap);
+    }
+};
 
 // One term of the Scatter Chain sum for the process count at index pidx: the gaps g(j m) for j
 // from the previous listed process count (1 before the first) up to P-1.  For a contiguous
 // range of P this is the single gap g((P-1) m); longer runs are added with compensation.
-// `i` carries the table interval from one call to the next (arguments must not decrease); pass
-// a negative value on the first call.
-__device__ __forceinline__ double s1_term(const double *s_tab, int npad, const GridDev &G, int pidx, double md, int &i)
+// The walk state must only see non-decreasing arguments.
+__device__ __forceinline__ double s1_term(const double *s_tab, int npad, const GridDev &G, int pidx, double md, GapWalk &w)
 {
     const int jhi = P_at(G, pidx) - 1;
     const int jlo = pidx == 0 ? 1 : P_at(G, pidx - 1);
-    if (i < 0) i = interval_of(s_tab, npad, static_cast<double>(jlo) * md);
-    if (jlo == jhi) return gap_walk(s_tab, npad, static_cast<double>(jlo) * md, i);
+    if (jlo == jhi) return w.at(s_tab, npad, static_cast<double>(jlo) * md);
     double sum = 0.0, comp = 0.0;
     for (int j = jlo; j <= jhi; ++j) {
-        const double y = gap_walk(s_tab, npad, static_cast<double>(j) * md, i) - comp;
+        const double y = w.at(s_tab, npad, static_cast<double>(j) * md) - comp;
         const double t = sum + y;
         comp = (t - sum) - y;
         sum = t;

@@ -104,6 +104,7 @@ constexpr int kMaxInlineS = 64;
 
 size_t fused_smem_bytes(const TableDev &T, const GridDev &G, bool inline_sweep);
 cudaError_t launch_fused(const FusedParams &p, bool predict, cudaStream_t st);
+cudaError_t launch_scatter(const FusedParams &p, cudaStream_t st);  // decision table, Scatter strategies only
 cudaError_t launch_sweep(const SweepParams &p, int n_tables_launch, cudaStream_t st);
 cudaError_t launch_s1_tiles(const S1Params &p, cudaStream_t st);
 size_t decide_smem_bytes(const TableDev &T, const GridDev &G);

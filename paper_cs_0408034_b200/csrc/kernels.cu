@@ -203,13 +203,11 @@ __global__ void __launch_bounds__(kThreads) s1_tile_sum_kernel(const S1Params p)
     __syncthreads();
 
     double acc = 0.0;
-    int walk = -1;
-    for (int pass = 0; pass < p.passes_per_tile; ++pass) {
-        const int p0 = (ptile * p.passes_per_tile + pass) * (kWarps * R) + warp * R;
-#pragma unroll
-        for (int r = 0; r < R; ++r)
-            if (p0 + r < p.G.n_P) acc += s1_term(s_tab, p.T.npad, p.G, p0 + r, md, walk);
-    }
+    GapWalk walk;
+    const int run_len = p.passes_per_tile * R;
+    const int p_warp = ptile * (kWarps * run_len) + warp * run_len;
+    for (int e = 0; e < run_len; ++e)
+        if (p_warp + e < p.G.n_P) acc += s1_term(s_tab, p.T.npad, p.G, p_warp + e, md, walk);
     s_red[warp * 32 + lane] = acc;
     __syncthreads();
     if (warp == 0 && midx < p.G.n_m) {
@@ -299,12 +297,17 @@ __global__ void __launch_bounds__(kThreads) fused_kernel(const FusedParams p)
     const double gm = gap_at(sm.tab, npad, md);
 
     // Scatter Binomial Tree: running sums of g(2^j m), j = 0..lc_max-1 (Table 2, third row)
-    if (warp == 0 && ((mask >> 12) & 1u)) {
-        double acc = 0.0, scale = 1.0;
-        for (int d = 0; d < p.G.lc_max; ++d) {
-            acc += gap_at(sm.tab, npad, md * scale);
-            sm.cum[d * 32 + lane] = acc;
-            scale *= 2.0;
+    // (the gaps are looked up by all warps, one j per warp at a time; warp 0 then adds them up)
+    if ((mask >> 12) & 1u) {
+        for (int d = warp; d < p.G.lc_max; d += kWarps)
+            sm.cum[d * 32 + lane] = gap_at(sm.tab, npad, md * static_cast<double>(1ull << d));
+        __syncthreads();
+        if (warp == 0) {
+            double acc = 0.0;
+            for (int d = 0; d < p.G.lc_max; ++d) {
+                acc += sm.cum[d * 32 + lane];
+                sm.cum[d * 32 + lane] = acc;
+            }
         }
     }
     // Inline candidate list: g(s) once per s, then the line coefficients per (s, m)
@@ -325,16 +328,30 @@ __global__ void __launch_bounds__(kThreads) fused_kernel(const FusedParams p)
     }
     __syncthreads();
 
-    double carry = 0.0;
-    int s1_walk = -1;  // table interval of this thread's last Scatter Chain argument
-    if (p.s1_carry) carry = p.s1_carry[(static_cast<size_t>(trel) * p.n_ptiles + ptile) * p.G.n_m + midx_c];
+    // Process counts of the tile: warp w owns the contiguous run [w * run_len, (w + 1) * run_len), R of them
+    // per pass, so that the Scatter Chain sum can run along a thread without a barrier per pass.
+    const int run_len = p.passes_per_tile * R;
+    const int p_warp = ptile * (kWarps * run_len) + warp * run_len;
+
+    // Scatter Chain: prefix of g(j m) in front of this thread's run = tile carry + the runs of the lower warps
+    double s1_run = 0.0;
+    GapWalk s1_walk;  // table interval of this thread's last Scatter Chain argument
+    if ((mask >> 11) & 1u) {
+        double mine = 0.0;
+        for (int e = 0; e < run_len; ++e)
+            if (p_warp + e < p.G.n_P) mine += s1_term(sm.tab, npad, p.G, p_warp + e, md, s1_walk);
+        sm.tot[warp * 32 + lane] = mine;
+        __syncthreads();
+        if (p.s1_carry) s1_run = p.s1_carry[(static_cast<size_t>(trel) * p.n_ptiles + ptile) * p.G.n_m + midx_c];
+        for (int w = 0; w < warp; ++w) s1_run += sm.tot[w * 32 + lane];
+        s1_walk.i = -1;
+    }
 
     const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
 
     for (int pass = 0; pass < p.passes_per_tile; ++pass) {
-        const int p_cta = (ptile * p.passes_per_tile + pass) * (kWarps * R);
-        if (p_cta >= p.G.n_P) break;  // uniform over the CTA
-        const int p0 = p_cta + warp * R;
+        const int p0 = p_warp + pass * R;
+        if (p0 >= p.G.n_P) break;  // this warp's run is exhausted (no barriers below)
 
         int Pv[R];
         bool ok[R];
@@ -346,29 +363,14 @@ __global__ void __launch_bounds__(kThreads) fused_kernel(const FusedParams p)
             pm1[r] = static_cast<double>(Pv[r] - 1);
         }
 
-        // ---- Scatter Chain: block scan of g(j m) over this pass's process counts ----
+        // ---- Scatter Chain: running sum of g(j m) along the thread's run ----
         double s1sum[R];
         if ((mask >> 11) & 1u) {
-            double run = 0.0;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                if (ok[r]) run += s1_term(sm.tab, npad, p.G, p0 + r, md, s1_walk);
-                s1sum[r] = run;
+                if (ok[r]) s1_run += s1_term(sm.tab, npad, p.G, p0 + r, md, s1_walk);
+                s1sum[r] = s1_run;
             }
-            double *tot = sm.tot + (pass & 1) * (kWarps * 32);
-            tot[warp * 32 + lane] = run;
-            __syncthreads();
-            double before = 0.0, all = 0.0;
-#pragma unroll
-            for (int w = 0; w < kWarps; ++w) {
-                const double v = tot[w * 32 + lane];
-                before += (w < warp) ? v : 0.0;
-                all += v;
-            }
-            const double base = carry + before;
-#pragma unroll
-            for (int r = 0; r < R; ++r) s1sum[r] += base;
-            carry += all;
         }
 
         // ---- running decision per cell (strict '<' in ascending id keeps the lowest id on ties) ----

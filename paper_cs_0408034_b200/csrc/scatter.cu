@@ -1,0 +1,194 @@
+// scatter_kernel: Scatter half of the decision table (Table 2 of the paper: Flat Tree, Chain,
+// Binomial Tree; selection as in Sections 1 and 5).
+//
+// Lanes are message sizes (32 consecutive m per warp, so every store is one aligned row segment);
+// each warp owns a contiguous run of process counts and walks it in ascending order, which turns
+// the Chain model's sum over j = 1..P-1 of g(j m) into a running sum along the thread: the argument
+// j m grows by m per step, the table interval is kept in registers and only reloaded when the
+// argument crosses a breakpoint.  The sum in front of a warp's run comes from the runs of the lower
+// warps (one pass over the run without stores, one barrier) plus the tile prefix computed by
+// s1_tile_sum_kernel / s1_tile_scan_kernel when the P range is split over several CTAs.
+#include "device_common.cuh"
+
+namespace plogp {
+
+namespace {
+
+// Interval walk without the clamp of gap_at: below the table a pseudo-interval with slope 0
+// holds g at its first value.
+struct LineWalk {
+    int i;
+    double key, next, slope, gap;
+
+    __device__ __forceinline__ void start(const double *s_tab, int npad, double x)
+    {
+        if (x < s_tab[0]) {
+            i = -1; key = 0.0; next = s_tab[0]; slope = 0.0; gap = s_tab[npad];
+        } else {
+            i = interval_of(s_tab, npad, x);
+            load(s_tab, npad);
+        }
+    }
+    __device__ __forceinline__ void load(const double *s_tab, int npad)
+    {
+        key = s_tab[i]; next = s_tab[i + 1]; slope = s_tab[2 * npad + i]; gap = s_tab[npad + i];
+    }
+    __device__ __forceinline__ double at(const double *s_tab, int npad, double x)
+    {
+        while (x >= next) { ++i; load(s_tab, npad); }
+        return fma(x - key, slope, gap);
+    }
+};
+
+}  // namespace
+
+// CONTIG: the process counts are the contiguous range P_lo + index (one new gap per step).
+template <bool CONTIG>
+__global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *s_tab = reinterpret_cast<double *>(smem_raw);
+    double *s_cum = s_tab + 3 * p.T.npad;      // [lc_max][32]
+    double *s_tot = s_cum + p.G.lc_max * 32;   // [kWarps][32]
+    const int npad = p.T.npad;
+    const uint32_t mask = p.G.mask;
+    const bool on10 = (mask >> 10) & 1u, on11 = (mask >> 11) & 1u, on12 = (mask >> 12) & 1u;
+
+    int b = blockIdx.x;
+    const int mtile = b % p.n_mtiles;
+    b /= p.n_mtiles;
+    const int ptile = b % p.n_ptiles;
+    const int trel = b / p.n_ptiles;
+    const int table = p.table0 + trel;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int midx = mtile * 32 + lane;
+    const bool m_ok = midx < p.G.n_m;
+    const int midx_c = min(midx, p.G.n_m - 1);
+    const double md = static_cast<double>(p.G.m_list[midx_c]);
+
+    stage_table(s_tab, p.T, table);
+    __syncthreads();
+    const double L = p.T.lat[table];
+    const double gm = gap_at(s_tab, npad, md);
+
+    // Binomial Tree: sums of g(2^j m); the gaps are looked up by all warps, warp 0 adds them up
+    if (on12) {
+        for (int d = warp; d < p.G.lc_max; d += kWarps)
+            s_cum[d * 32 + lane] = gap_at(s_tab, npad, md * static_cast<double>(1ull << d));
+        __syncthreads();
+        if (warp == 0) {
+            double acc = 0.0;
+            for (int d = 0; d < p.G.lc_max; ++d) {
+                acc += s_cum[d * 32 + lane];
+                s_cum[d * 32 + lane] = acc;
+            }
+        }
+    }
+
+    // this warp's run of process-count indices
+    const int run_len = p.passes_per_tile * kFusedR;
+    const int e0 = ptile * (kWarps * run_len) + warp * run_len;
+    const int e1 = min(e0 + run_len, p.G.n_P);
+
+    // One step of the Chain sum: all gaps g(j m) with j from the previous process count (1 before
+    // the first) to P-1; a single gap when the process counts are contiguous.
+    auto chain_step = [&](int e, int P, LineWalk &w, double &x) -> double {
+        if (CONTIG && e > 0) {
+            const double g = w.at(s_tab, npad, x);
+            x += md;  // exact: j m < 2^53
+            return g;
+        }
+        const int jlo = e == 0 ? 1 : P_at(p.G, e - 1);
+        double sum = 0.0, comp = 0.0;
+        for (int j = jlo; j <= P - 1; ++j) {
+            const double y = w.at(s_tab, npad, static_cast<double>(j) * md) - comp;
+            const double t = sum + y;
+            comp = (t - sum) - y;
+            sum = t;
+        }
+        x = static_cast<double>(P) * md;
+        return sum;
+    };
+    auto first_arg = [&](int e) {  // smallest j m that the run starting at index e will look up
+        const int jlo = e == 0 ? 1 : P_at(p.G, e - 1);
+        return static_cast<double>(jlo) * md;
+    };
+
+    double run = 0.0;
+    if (on11) {
+        double mine = 0.0;
+        if (e0 < e1) {
+            LineWalk w;
+            double x = first_arg(e0);
+            w.start(s_tab, npad, x);
+            for (int e = e0; e < e1; ++e) mine += chain_step(e, P_at(p.G, e), w, x);
+        }
+        s_tot[warp * 32 + lane] = mine;
+    }
+    __syncthreads();  // also publishes s_cum
+    if (on11) {
+        if (p.s1_carry) run = p.s1_carry[(static_cast<size_t>(trel) * p.n_ptiles + ptile) * p.G.n_m + midx_c];
+        for (int w = 0; w < warp; ++w) run += s_tot[w * 32 + lane];
+    }
+    if (e0 >= e1) return;
+
+    LineWalk w;
+    double x = first_arg(e0);
+    if (on11) w.start(s_tab, npad, x);
+
+    const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
+    size_t o = (static_cast<size_t>(table) * 2 + 1) * plane + static_cast<size_t>(e0) * p.G.n_m + midx;
+    int P = P_at(p.G, e0);
+    int lc = 32 - __clz(P - 1);               // ceil(log2 P)
+    double lcL = static_cast<double>(lc) * L;
+    double s2 = on12 ? s_cum[(lc - 1) * 32 + lane] + lcL : 0.0;
+    double pm1 = static_cast<double>(P - 1);
+
+    for (int e = e0; e < e1; ++e) {
+        if (!CONTIG || e == e0) {
+            P = P_at(p.G, e);
+            pm1 = static_cast<double>(P - 1);
+        }
+        if (32 - __clz(P - 1) != lc) {  // P passed a power of two
+            lc = 32 - __clz(P - 1);
+            lcL = static_cast<double>(lc) * L;
+            if (on12) s2 = s_cum[(lc - 1) * 32 + lane] + lcL;
+        }
+        double bt = CUDART_INF;
+        int bid = 255;
+        if (on10) { bt = fma(pm1, gm, L); bid = 10; }                    // Flat Tree
+        if (on11) {                                                      // Chain
+            run += chain_step(e, P, w, x);
+            const double t = fma(pm1, L, run);
+            if (t < bt) { bt = t; bid = 11; }
+        }
+        if (on12 && s2 < bt) { bt = s2; bid = 12; }                      // Binomial Tree
+        if (m_ok) {
+            p.d_time[o] = bt;
+            p.d_strategy[o] = static_cast<uint8_t>(bid);
+            p.d_sbytes[o] = 0u;
+        }
+        o += p.G.n_m;
+        if (CONTIG) { ++P; pm1 += 1.0; }
+    }
+}
+
+cudaError_t launch_scatter(const FusedParams &p, cudaStream_t st)
+{
+    const size_t smem = (3 * static_cast<size_t>(p.T.npad) + static_cast<size_t>(p.G.lc_max) * 32 + kWarps * 32) * sizeof(double);
+    const long long blocks = static_cast<long long>(p.n_mtiles) * p.n_ptiles * p.n_tables_launch;
+    if (blocks <= 0 || blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    cudaError_t e = cudaSuccess;
+    if (p.G.P_list == nullptr) {
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(scatter_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        scatter_kernel<true><<<static_cast<unsigned>(blocks), kThreads, smem, st>>>(p);
+    } else {
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(scatter_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        scatter_kernel<false><<<static_cast<unsigned>(blocks), kThreads, smem, st>>>(p);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace plogp
