@@ -52,16 +52,37 @@ def make_workload(name: str, scale: str, rank: int):
 
 
 def work_counts(w):
-    """Cells and the algorithmic work of one step (per segmented cell one DFMA and
-    one compare, per unsegmented cell one DFMA; bytes = the decision table written once)."""
+    """Cells of one step and the algorithmic work of each kernel: a segmented cell
+    is one DFMA and one compare (2 FP64 issue slots), an unsegmented cell one DFMA, a Scatter Chain
+    element one interpolation DFMA, one running-sum DADD and the model's DFMA; HBM bytes are the decision
+    table written once (13 B per decision cell)."""
     mask = w.strategy_mask
-    n_seg = sum((mask >> b) & 1 for b in (2, 5, 9))
-    n_unseg = sum((mask >> b) & 1 for b in range(13)) - n_seg
-    seg_cells = w.n_tables * w.n_P * n_seg * int(w.n_candidates().sum())
-    unseg_cells = w.n_tables * w.n_P * n_unseg * w.n_m
-    dec = w.decision_cells()
-    return {"model_cells": seg_cells + unseg_cells, "segmented_cells": seg_cells, "decision_cells": dec,
-            "fp64_slots": 2 * seg_cells + unseg_cells, "hbm_bytes": 13 * dec}
+    seg_ids = [b for b in (2, 5, 9) if (mask >> b) & 1]
+    unseg_b = [b for b in (0, 1, 3, 4, 6, 7, 8) if (mask >> b) & 1]
+    scat = [b for b in (10, 11, 12) if (mask >> b) & 1]
+    cells_pm = w.n_tables * w.n_P * w.n_m
+    seg_cells = w.n_tables * w.n_P * len(seg_ids) * int(w.n_candidates().sum())
+    bcast_dec = cells_pm if (seg_ids or unseg_b) else 0
+    scat_dec = cells_pm if scat else 0
+    scat_slots = cells_pm * (((mask >> 10) & 1) + 3 * ((mask >> 11) & 1) + ((mask >> 12) & 1))
+    long_lists = bool(seg_ids) and len(w.s_values()) > 64
+    per_kernel = {}
+    if long_lists:
+        per_kernel["sweep_kernel"] = {"fp64_slots": 2 * seg_cells, "hbm_bytes": 0}
+        per_kernel["fused_kernel"] = {"fp64_slots": len(unseg_b) * cells_pm + scat_slots, "hbm_bytes": 13 * (bcast_dec + scat_dec)}
+    else:
+        if seg_ids:
+            per_kernel["decide_kernel"] = {"fp64_slots": 2 * seg_cells + len(unseg_b) * cells_pm, "hbm_bytes": 13 * bcast_dec}
+            if scat:
+                per_kernel["scatter_kernel"] = {"fp64_slots": scat_slots, "hbm_bytes": 13 * scat_dec}
+        elif unseg_b:
+            per_kernel["fused_kernel"] = {"fp64_slots": len(unseg_b) * cells_pm + scat_slots, "hbm_bytes": 13 * (bcast_dec + scat_dec)}
+        elif scat:
+            per_kernel["scatter_kernel"] = {"fp64_slots": scat_slots, "hbm_bytes": 13 * scat_dec}
+    total_slots = sum(k["fp64_slots"] for k in per_kernel.values())
+    return {"model_cells": seg_cells + (len(unseg_b) + len(scat)) * cells_pm, "segmented_cells": seg_cells,
+            "decision_cells": bcast_dec + scat_dec, "fp64_slots": total_slots, "hbm_bytes": 13 * (bcast_dec + scat_dec),
+            "per_kernel": per_kernel}
 
 
 class ClockSampler:
@@ -116,6 +137,17 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(s[0] for s in self.samples), "sm_max_mhz": self.sm_max,
                 "reasons": [k for k, bit in names.items() if seen & bit],
                 "power_w_max": max(s[1] for s in self.samples), "samples": len(self.samples)}
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    """Largest value over all ranks (timings of a multi-GPU run are the slowest rank's)."""
+    if world == 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
 
 
 def measured_peaks():
@@ -237,6 +269,7 @@ def main():
     if not uuid.startswith("GPU-"):
         uuid = "GPU-" + uuid
     launches0 = plogp.kernel_launches()
+    plogp.profile_enable(tabs, True)
     events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     with ClockSampler(uuid) as clocks:
         barrier()
@@ -248,11 +281,10 @@ def main():
                 flush.fill_(1)
         barrier()
     launches = plogp.kernel_launches() - launches0
+    kernel_ms = plogp.profile_read(tabs)   # {kernel: (ms over the timed region, launches)}
+    plogp.profile_enable(tabs, False)
     total_ms = sum(a.elapsed_time(b) for a, b in events)
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, "cuda")
     ms_per_step = total_ms / args.steps
 
     # ---- end to end through the public API with host buffers ----
@@ -277,10 +309,7 @@ def main():
             e2e_step()
         barrier()
         e2e_ms = (time.perf_counter() - t0) * 1e3 / args.e2e_steps
-        if world > 1:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
         del host
 
     if rank != 0:
@@ -290,23 +319,40 @@ def main():
 
     fma_rate = plogp.fp64_fma_rate(100.0)
     hbm_gbs, peak_src = measured_peaks()
+    step_s = ms_per_step * 1e-3
+
+    def roof(name, ms_total, n_launch):
+        """Roofline of one kernel: algorithmic work per launch / its average launch duration (CUDA events
+        recorded by the library on the launching stream during the timed region)."""
+        work = counts["per_kernel"].get(name)
+        if work is None or n_launch == 0:
+            return {"kernel": name, "launches": n_launch, "ms_total": ms_total}
+        per_launch = args.steps / n_launch  # a kernel launched once per step does one step's work
+        dur = ms_total / n_launch * 1e-3
+        slots, nbytes = work["fp64_slots"] * per_launch, work["hbm_bytes"] * per_launch
+        t_alu, t_hbm = slots / fma_rate, nbytes / (hbm_gbs * 1e9)
+        alu = t_alu >= t_hbm
+        return {"kernel": name, "launches": n_launch, "ms_total": ms_total, "avg_ms": dur * 1e3,
+                "bound": "alu" if alu else "hbm",
+                "achieved": slots / dur / 1e12 if alu else nbytes / dur / 1e9,
+                "peak": fma_rate / 1e12 if alu else hbm_gbs,
+                "unit": "T FP64 thread-instr/s" if alu else "GB/s",
+                "frac": max(t_alu, t_hbm) / dur,
+                "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
+                "peak_source": ("DFMA issue rate measured in this run by plogp_fp64_fma_rate, of measured (nominal %.2f T/s = 148 SMs x 64 lanes x 1.965 GHz)"
+                                % (NOMINAL_FP64_FMA_RATE / 1e12)) if alu else "HBM copy bandwidth, of %s" % peak_src}
+
+    kernels = [roof(k, v[0], v[1]) for k, v in kernel_ms.items()]
+    tot_kernel_ms = sum(k["ms_total"] for k in kernels) or 1.0
+    for k in kernels:
+        k["share"] = k["ms_total"] / tot_kernel_ms
+    dominant = max(kernels, key=lambda k: k["ms_total"]) if kernels else {}
+    roofline = dict(dominant)
+    roofline["traffic"] = None
     t_alu = counts["fp64_slots"] / fma_rate
     t_hbm = counts["hbm_bytes"] / (hbm_gbs * 1e9)
-    step_s = ms_per_step * 1e-3
-    alu_bound = t_alu >= t_hbm
-    roofline = {
-        "bound": "alu" if alu_bound else "hbm",
-        "achieved": counts["fp64_slots"] / step_s / 1e12 if alu_bound else counts["hbm_bytes"] / step_s / 1e9,
-        "peak": fma_rate / 1e12 if alu_bound else hbm_gbs,
-        "unit": "T FP64 thread-instr/s" if alu_bound else "GB/s",
-        "frac": max(t_alu, t_hbm) / step_s,
-        "traffic": None,
-        "peak_source": ("DFMA issue rate measured in this run by plogp_fp64_fma_rate (nominal %.2f T/s)" % (NOMINAL_FP64_FMA_RATE / 1e12))
-        if alu_bound else "%s HBM copy bandwidth" % peak_src,
-        "kernel": "sweep_kernel+fused_kernel (step)" if args.workload == "cfg3" else "fused_kernel",
-        "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
-        "hbm_achieved_gbs": counts["hbm_bytes"] / step_s / 1e9, "hbm_peak_gbs": hbm_gbs, "hbm_peak_source": peak_src,
-    }
+    roofline["step"] = {"frac": max(t_alu, t_hbm) / step_s, "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
+                        "note": "whole step (all kernels) against max(FP64 issue, HBM bytes)"}
 
     line = {
         "metric": "model_cells_per_sec", "value": world * counts["model_cells"] / step_s, "unit": "cells/s",
@@ -323,6 +369,7 @@ def main():
                 "ms_per_step": e2e_ms, "steps": args.e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
         "roofline": roofline,
+        "kernels": kernels,
     }
     if world == 1 and not args.no_cpu_baseline:
         v, cores, text = oracle_sample_rate(w, 15.0)

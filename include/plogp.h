@@ -167,6 +167,25 @@ int plogp_scatter_chain_static(int n_bp, const uint64_t *d_sizes_bytes, const do
                                int32_t P_lo, int32_t P_hi, const uint64_t *d_m_bytes, int32_t n_m,
                                double *d_time, void *stream);
 
+/*
+ * Per-kernel device timing (measurement aid, no counterpart in the paper).  While enabled, every
+ * kernel that plogp_predict / plogp_select_best launch on this handle is bracketed by two CUDA
+ * events recorded on the caller's stream.  plogp_profile_read waits for the recorded events,
+ * adds the elapsed milliseconds and launch counts per kernel kind into ms[PLOGP_N_KERNEL_KINDS] and
+ * launches[PLOGP_N_KERNEL_KINDS] (HOST arrays), and forgets them.  Read (or free the handle)
+ * regularly: each launch keeps two events alive until then.
+ */
+enum {
+    PLOGP_KERNEL_SWEEP = 0,        /* segment sweep over long candidate lists */
+    PLOGP_KERNEL_CHAIN_PREFIX = 1, /* Scatter Chain tile sums + their scan (two launches, timed together) */
+    PLOGP_KERNEL_FUSED = 2,        /* all strategies, lanes <-> m (predictions, long lists' final pass) */
+    PLOGP_KERNEL_DECIDE = 3,       /* Broadcast decision, lanes <-> P (short candidate lists) */
+    PLOGP_KERNEL_SCATTER = 4,      /* Scatter decision */
+    PLOGP_N_KERNEL_KINDS = 5
+};
+int plogp_profile_enable(plogp_tables *tables, int enable);
+int plogp_profile_read(plogp_tables *tables, double *ms, int32_t *launches);
+
 /* Number of kernels this library has launched in the calling process so far (all handles, all
  * threads).  Bookkeeping for benchmarks; no counterpart in the paper. */
 uint64_t plogp_kernel_launches(void);

@@ -77,9 +77,38 @@ struct plogp_tables {
     unsigned char *d_ws = nullptr;
     size_t ws_cap = 0;
     Plan plan;
+    // optional per-kernel timing: event pairs recorded around every launch while enabled
+    bool profiling = false;
+    struct Timed { int kind; cudaEvent_t a, b; };
+    std::vector<Timed> timed;
 };
 
 namespace {
+
+// Brackets one kernel launch with events on the caller's stream when timing is enabled.
+struct LaunchTimer {
+    plogp_tables *h;
+    cudaStream_t st;
+    cudaEvent_t a = nullptr, b = nullptr;
+    int kind;
+    LaunchTimer(plogp_tables *h_, int kind_, cudaStream_t st_) : h(h_), st(st_), kind(kind_)
+    {
+        if (!h->profiling) return;
+        if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess || cudaEventRecord(a, st) != cudaSuccess) {
+            if (a) cudaEventDestroy(a);
+            if (b) cudaEventDestroy(b);
+            a = b = nullptr;
+            cudaGetLastError();
+        }
+    }
+    ~LaunchTimer()
+    {
+        if (!a) return;
+        if (cudaEventRecord(b, st) == cudaSuccess) h->timed.push_back({kind, a, b});
+        else { cudaEventDestroy(a); cudaEventDestroy(b); cudaGetLastError(); }
+    }
+};
+
 
 template <typename V>
 void put(std::vector<unsigned char> &buf, const V &v)
@@ -357,7 +386,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             sp.pair_row = reinterpret_cast<const int32_t *>(h->d_grid + pl.off_pair_row);
             sp.n_pairs = pl.n_pairs; sp.n_ptiles = pl.sweep_ptiles; sp.chunk_len = pl.chunk_len;
             sp.part_time = part_time; sp.part_idx = part_idx; sp.n_seg = pl.n_seg; sp.table0 = t0;
-            CK(launch_sweep(sp, nt, st));
+            { LaunchTimer lt(h, PLOGP_KERNEL_SWEEP, st); CK(launch_sweep(sp, nt, st)); }
             g_launches += 1;
         }
         if (need_carry) {
@@ -365,7 +394,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             s.T = h->T; s.G = pl.G;
             s.n_mtiles = pl.n_mtiles; s.n_ptiles = n_ptiles; s.passes_per_tile = passes_per_tile;
             s.table0 = t0; s.n_tables_launch = nt; s.tile_sum = tile_sum;
-            CK(launch_s1_tiles(s, st));
+            { LaunchTimer lt(h, PLOGP_KERNEL_CHAIN_PREFIX, st); CK(launch_s1_tiles(s, st)); }
             g_launches += 2;
         }
         GridDev Gf = pl.G;
@@ -377,7 +406,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             dp.n_mgroups = pl.dec_mgroups; dp.n_ptiles = pl.dec_ptiles;
             dp.table0 = t0; dp.n_tables_launch = nt;
             dp.d_strategy = out.d_strategy; dp.d_sbytes = out.d_sbytes; dp.d_time = out.d_time;
-            CK(launch_decide(dp, st));
+            { LaunchTimer lt(h, PLOGP_KERNEL_DECIDE, st); CK(launch_decide(dp, st)); }
             g_launches += 1;
             Gf.mask &= 0x1C00u;
             Gf.n_s = 0;
@@ -393,8 +422,8 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
         fp.part_idx = part_idx;
         fp.pair_base = pl.inline_sweep ? nullptr : reinterpret_cast<const int32_t *>(h->d_grid + pl.off_pair_base);
         fp.n_pairs = pl.n_pairs; fp.n_seg = pl.n_seg;
-        if (!predict && (Gf.mask & 0x3FFu) == 0) CK(launch_scatter(fp, st));
-        else CK(launch_fused(fp, predict, st));
+        if (!predict && (Gf.mask & 0x3FFu) == 0) { LaunchTimer lt(h, PLOGP_KERNEL_SCATTER, st); CK(launch_scatter(fp, st)); }
+        else { LaunchTimer lt(h, PLOGP_KERNEL_FUSED, st); CK(launch_fused(fp, predict, st)); }
         g_launches += 1;
     }
     return PLOGP_OK;
@@ -478,7 +507,33 @@ int plogp_table_free(plogp_tables *h)
             if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree");
         }
     }
+    for (auto &t : h->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
     delete h;
+    return rc;
+}
+
+int plogp_profile_enable(plogp_tables *h, int enable)
+{
+    if (!h) return PLOGP_E_INVAL;
+    h->profiling = enable != 0;
+    return PLOGP_OK;
+}
+
+int plogp_profile_read(plogp_tables *h, double *ms, int32_t *launches)
+{
+    if (!h || !ms || !launches) return PLOGP_E_INVAL;
+    for (int k = 0; k < PLOGP_N_KERNEL_KINDS; ++k) { ms[k] = 0.0; launches[k] = 0; }
+    int rc = PLOGP_OK;
+    for (auto &t : h->timed) {
+        float v = 0.f;
+        cudaError_t e = cudaEventSynchronize(t.b);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&v, t.a, t.b);
+        if (e == cudaSuccess) { ms[t.kind] += v; launches[t.kind] += 1; }
+        else rc = cuda_fail(e, "cudaEventElapsedTime");
+        cudaEventDestroy(t.a);
+        cudaEventDestroy(t.b);
+    }
+    h->timed.clear();
     return rc;
 }
 

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libplogp.so")
 N_STRATEGIES = 13
 SEGMENTED_IDS = (2, 5, 9)
 EXPORTS = ("plogp_table_load", "plogp_table_free", "plogp_predict", "plogp_select_best",
-           "plogp_status_string", "plogp_last_cuda_error", "plogp_kernel_launches", "plogp_fp64_fma_rate",
+           "plogp_status_string", "plogp_last_cuda_error", "plogp_kernel_launches", "plogp_fp64_fma_rate", "plogp_profile_enable", "plogp_profile_read",
            "plogp_scatter_chain_static")
 
 OK, E_INVAL, E_NOMEM, E_CUDA, E_RANGE = 0, -1, -2, -3, -4
@@ -58,6 +58,10 @@ lib.plogp_last_cuda_error.argtypes = []
 lib.plogp_scatter_chain_static.restype = C.c_int
 lib.plogp_scatter_chain_static.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_double, C.c_int32, C.c_int32,
                                            C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+lib.plogp_profile_enable.restype = C.c_int
+lib.plogp_profile_enable.argtypes = [C.c_void_p, C.c_int]
+lib.plogp_profile_read.restype = C.c_int
+lib.plogp_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int32)]
 lib.plogp_kernel_launches.restype = C.c_uint64
 lib.plogp_kernel_launches.argtypes = []
 lib.plogp_fp64_fma_rate.restype = C.c_double
@@ -248,3 +252,19 @@ def scatter_chain_static(d_sizes, d_gap, latency: float, P_lo: int, P_hi: int, d
                                           int(P_lo), int(P_hi), d_m.data_ptr(), int(d_m.numel()), out.data_ptr(),
                                           _stream_ptr(stream)), "plogp_scatter_chain_static")
     return out
+
+
+KERNEL_KINDS = ("sweep_kernel", "s1_tile_sum_kernel+s1_tile_scan_kernel", "fused_kernel", "decide_kernel", "scatter_kernel")
+
+
+def profile_enable(tables: Tables, enable: bool = True) -> None:
+    """``plogp_profile_enable``: record CUDA events around every kernel launched on this handle."""
+    _check(lib.plogp_profile_enable(tables.handle, int(enable)), "plogp_profile_enable")
+
+
+def profile_read(tables: Tables) -> dict:
+    """``plogp_profile_read``: {kernel kind: (milliseconds, launches)} since the last read."""
+    ms = (C.c_double * len(KERNEL_KINDS))()
+    n = (C.c_int32 * len(KERNEL_KINDS))()
+    _check(lib.plogp_profile_read(tables.handle, ms, n), "plogp_profile_read")
+    return {k: (ms[i], n[i]) for i, k in enumerate(KERNEL_KINDS) if n[i]}
