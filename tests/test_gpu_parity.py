@@ -131,3 +131,58 @@ def test_single_cell_and_two_breakpoints(plogp):
     np.testing.assert_allclose(pred.time[0, :, 0, 0].cpu().numpy(), o.time[:, 0, 0], rtol=1e-12)
     od = po.select_grid(wl.ALL_STRATEGIES, o)
     assert dec.strategy[0, :, 0, 0].tolist() == od.strategy[:, 0, 0].tolist()
+
+
+def test_config4_full_size_sampled_tables(plogp):
+    """The benchmark's launch configuration (4096 tables, decide_kernel + scatter_kernel); whole decision
+    tables of sampled networks, first / middle / last, are compared with the oracle."""
+    import torch
+    w = wl.config4()
+    ot = {t: None for t in (0, 1, 777, 2048, 4095)}
+    from oracle import plogp_oracle as po
+    for t in ot:
+        ot[t] = po.Table(w.table_sizes(t), w.gaps[t], w.latency[t])
+    with plogp.Tables.from_workload(w) as tabs:
+        dec = plogp.select_best(tabs, w)
+        torch.cuda.synchronize()
+        n = check_decision(w, ot, dec, tables=list(ot))
+    assert n == len(ot) * 2 * w.n_P * w.n_m
+    # every cell of every table was written, with an eligible id
+    assert int((dec.strategy[:, 0] > 9).sum()) == 0 and int(((dec.strategy[:, 1] < 10) | (dec.strategy[:, 1] > 12)).sum()) == 0
+    assert bool(torch.isfinite(dec.time).all())
+
+
+def test_config3_full_size_sampled_cells(plogp):
+    """The exhaustive sweep at full size (262144 candidates, P up to 4096) in the benchmark's launch
+    configuration; the oracle re-searches sampled (P, m) cells one by one."""
+    import torch
+    from oracle import plogp_oracle as po
+    from parity import _check_seg, oracle_sgrid, TIME_RTOL
+    w = wl.config3()
+    t = oracle_tables(w)[0]
+    sg = oracle_sgrid(w)
+    with plogp.Tables.from_workload(w) as tabs:
+        pred = plogp.predict(tabs, w)
+        dec = plogp.select_best(tabs, w)
+        torch.cuda.synchronize()
+    p_idx = [0, 1, 2, 30, 31, 32, 255, 256, 257, 1000, 2047, 2048, 2049, 3000, 4093, 4094]
+    m_idx = [0, 1, 40, 63, 64, 90, 126, 127]
+    time = pred.time[0].cpu().numpy()
+    best = pred.best_s[0].cpu().numpy().view(np.uint32)
+    d_id, d_s, d_t = (x[0, 0].cpu().numpy() for x in (dec.strategy, dec.s_bytes, dec.time))
+    for ip in p_idx:
+        for im in m_idx:
+            P, m = int(w.P_values()[ip]), int(w.m[im])
+            res = {}
+            for q, sid in ((0, 2), (1, 5)):
+                s, v, ru = po.segment_search(t, sid, P, m, sg, w.k_mode)
+                res[sid] = _check_seg(w, t, sid, P, m, int(best[q, ip, im]), time[sid, ip, im], s, v, ru,
+                                      "id %d P %d m %d" % (sid, P, m))
+            # decision: the cheaper of the two (id 2 on ties)
+            sid = int(d_id[ip, im])
+            assert sid in (2, 5)
+            other = 5 if sid == 2 else 2
+            assert abs(d_t[ip, im] - time[sid, ip, im]) <= TIME_RTOL * d_t[ip, im]
+            assert d_t[ip, im] <= time[other, ip, im] * (1 + 1e-9)
+            assert int(np.uint32(d_s[ip, im])) == int(best[(2, 5).index(sid), ip, im])
+    assert np.isnan(time[[0, 1, 3, 4, 6, 7, 8, 9, 10, 11, 12]]).all()
