@@ -187,13 +187,17 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 }
                 for (int chunk = 0; chunk < n_chunks; ++chunk) {
                     if (chunk == cp) continue;
-                    bool any = false;
+                    // one flag per cell: a single flag would chain all 16 integer compares through one predicate
+                    bool f[R];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) f[r] = false;
 #pragma unroll
                     for (int u = 0; u < U; ++u) {
 #pragma unroll
                         for (int r = 0; r < R; ++r)
-                            any |= __double2hiint(eval(r, chunk * U + u)) <= __double2hiint(st[r]);
+                            f[r] |= __double2hiint(eval(r, chunk * U + u)) <= __double2hiint(st[r]);
                     }
+                    const bool any = (f[0] | f[1]) | (f[2] | f[3]);
                     if (any) {  // exact pass; candidates arrive out of order, so ties go to the smaller index
 #pragma unroll 1
                         for (int u = 0; u < U; ++u) {

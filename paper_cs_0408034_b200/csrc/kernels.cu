@@ -99,28 +99,39 @@ __global__ void __launch_bounds__(kThreads, 2) sweep_kernel(const SweepParams p)
             // Hot path: every cell is evaluated (one DFMA); the comparison with the running minimum is
             // first taken on the high words only, in the integer pipe.  Times are non-negative, so the
             // high word of a smaller double is never larger: a cell can only improve if that test holds.
-            bool any5 = false, any2 = false, any9 = false;
+            // (one flag per register cell: a single flag would chain all the integer compares of the
+            // chunk through one predicate, and that dependent chain, not a pipe, then sets the pace)
+            bool f5[R], f2[R], f9[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) f5[r] = f2[r] = f9[r] = false;
 #pragma unroll
             for (int u = 0; u < kSweepU; ++u) {
                 if (HAS5) {
                     const double2 c = bc[i + u];
 #pragma unroll
                     for (int r = 0; r < R; ++r)
-                        any5 |= __double2hiint(fma(pm1[r], c.x, c.y)) <= __double2hiint(best5[r]);
+                        f5[r] |= __double2hiint(fma(pm1[r], c.x, c.y)) <= __double2hiint(best5[r]);
                 }
                 if (HAS2 || HAS9) {
                     const double q = qq[i + u];
                     if (HAS2) {
 #pragma unroll
                         for (int r = 0; r < R; ++r)
-                            any2 |= __double2hiint(fma(pm1[r], q, L)) <= __double2hiint(best2[r]);
+                            f2[r] |= __double2hiint(fma(pm1[r], q, L)) <= __double2hiint(best2[r]);
                     }
                     if (HAS9) {
 #pragma unroll
                         for (int r = 0; r < R; ++r)
-                            any9 |= __double2hiint(fma(lf[r], q, lcL[r])) <= __double2hiint(best9[r]);
+                            f9[r] |= __double2hiint(fma(lf[r], q, lcL[r])) <= __double2hiint(best9[r]);
                     }
                 }
+            }
+            bool any5 = false, any2 = false, any9 = false;
+#pragma unroll
+            for (int r = 0; r < R; r += 2) {
+                any5 |= f5[r] | f5[r + 1];
+                any2 |= f2[r] | f2[r + 1];
+                any9 |= f9[r] | f9[r + 1];
             }
             // Exact passes over the same candidates, in ascending order, strict '<' (smallest s on ties).
             if (HAS5 && any5) {
