@@ -170,7 +170,9 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 return static_cast<int>(__reduce_min_sync(0xffffffffu, key) & 63u) / U;
             };
             // Segmented model reduced over the candidates: eval(r, cand) is the model cell.
-            auto segmented = [&](int id, int cp, auto eval) {
+            // Segmented model reduced over the candidates: load(cand) fetches the candidate's line
+            // coefficients from shared memory, eval(r, coef) is the model cell.
+            auto segmented = [&](int id, int cp, auto load, auto eval) {
                 double st[R];
                 uint32_t si[R];
 #pragma unroll
@@ -179,14 +181,23 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
 #pragma unroll 1
                 for (int u = 0; u < U; ++u) {
                     const uint32_t cand = cp * U + u;
+                    const auto k = load(cand);
 #pragma unroll
                     for (int r = 0; r < R; ++r) {
-                        const double t = eval(r, cand);
+                        const double t = eval(r, k);
                         if (t < st[r]) { st[r] = t; si[r] = cand; }
                     }
                 }
-                for (int chunk = 0; chunk < n_chunks; ++chunk) {
-                    if (chunk == cp) continue;
+                // all other chunks; the next chunk's coefficients are fetched before the current one is tested
+                decltype(load(0)) cur[U], nxt[U];
+                int chunk = cp == 0 ? 1 : 0;
+#pragma unroll
+                for (int u = 0; u < U; ++u) cur[u] = load(min(chunk, n_chunks - 1) * U + u);
+                while (chunk < n_chunks) {
+                    int next = chunk + 1;
+                    next += next == cp;
+#pragma unroll
+                    for (int u = 0; u < U; ++u) nxt[u] = load(min(next, n_chunks - 1) * U + u);
                     // one flag per cell: a single flag would chain all 16 integer compares through one predicate
                     bool f[R];
 #pragma unroll
@@ -195,20 +206,22 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                     for (int u = 0; u < U; ++u) {
 #pragma unroll
                         for (int r = 0; r < R; ++r)
-                            f[r] |= __double2hiint(eval(r, chunk * U + u)) <= __double2hiint(st[r]);
+                            f[r] |= __double2hiint(eval(r, cur[u])) <= __double2hiint(st[r]);
                     }
-                    const bool any = (f[0] | f[1]) | (f[2] | f[3]);
-                    if (any) {  // exact pass; candidates arrive out of order, so ties go to the smaller index
-#pragma unroll 1
+                    if ((f[0] | f[1]) | (f[2] | f[3])) {  // exact pass; chunks arrive out of order: ties go to the smaller index
+#pragma unroll
                         for (int u = 0; u < U; ++u) {
                             const uint32_t cand = chunk * U + u;
 #pragma unroll
                             for (int r = 0; r < R; ++r) {
-                                const double t = eval(r, cand);
+                                const double t = eval(r, cur[u]);
                                 if (t < st[r] || (t == st[r] && cand < si[r])) { st[r] = t; si[r] = cand; }
                             }
                         }
                     }
+#pragma unroll
+                    for (int u = 0; u < U; ++u) cur[u] = nxt[u];
+                    chunk = next;
                 }
                 if (ns == 0) {
 #pragma unroll
@@ -232,7 +245,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 consider(1, v, nullptr);
             }
             if ((mask >> 2) & 1u)  // Segmented Flat Tree
-                segmented(2, cpQ, [&](int r, int cand) { return fma(pm1[r], sm.cQ[cand], L); });
+                segmented(2, cpQ, [&](int cand) { return sm.cQ[cand]; }, [&](int r, double q) { return fma(pm1[r], q, L); });
             if ((mask >> 3) & 1u) {  // Chain
 #pragma unroll
                 for (int r = 0; r < R; ++r) v[r] = pm1[r] * (gm + L);
@@ -245,7 +258,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             }
             if ((mask >> 5) & 1u) {  // Segmented Chain
                 const int cp5 = pilot_chunk([&](int cand) { const double2 c = sm.cBC[cand]; return fma(pm1_mid, c.x, c.y); });
-                segmented(5, cp5, [&](int r, int cand) { const double2 c = sm.cBC[cand]; return fma(pm1[r], c.x, c.y); });
+                segmented(5, cp5, [&](int cand) { return sm.cBC[cand]; }, [&](int r, double2 c) { return fma(pm1[r], c.x, c.y); });
             }
             if ((mask >> 6) & 1u) {  // Binary Tree (the printed bound)
 #pragma unroll
@@ -263,7 +276,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 consider(8, v, nullptr);
             }
             if ((mask >> 9) & 1u)  // Segmented Binomial Tree
-                segmented(9, cpQ, [&](int r, int cand) { return fma(lf[r], sm.cQ[cand], lcL[r]); });
+                segmented(9, cpQ, [&](int cand) { return sm.cQ[cand]; }, [&](int r, double q) { return fma(lf[r], q, lcL[r]); });
 
 #pragma unroll
             for (int r = 0; r < R; ++r) {
