@@ -30,6 +30,11 @@ if ROOT not in sys.path:
 from paper_cs_0408034_b200 import workloads as wl  # noqa: E402
 
 NOMINAL_FP64_FMA_RATE = 148 * 64 * 1.965e9  # SMs x FP64 lanes per SM x max SM clock
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
+# (reduced cfg4 with 256 tables; output bytes grow in proportion to the table count, so a full launch of
+# 4096 tables is 16 x the captured one).  Set an entry to None when its kernel changes after the capture.
+NCU_TRAFFIC_BYTES_PER_TABLE = {"decide_kernel": (162.75e6 + 0.45e6) / 256, "scatter_kernel": (158.83e6 + 0.94e6) / 256,
+                               "sweep_kernel": None}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -348,7 +353,9 @@ def main():
         k["share"] = k["ms_total"] / tot_kernel_ms
     dominant = max(kernels, key=lambda k: k["ms_total"]) if kernels else {}
     roofline = dict(dominant)
-    roofline["traffic"] = None
+    per_table = NCU_TRAFFIC_BYTES_PER_TABLE.get(dominant.get("kernel"))
+    roofline["traffic"] = per_table * w.n_tables if (per_table and args.workload == "cfg4") else None
+    roofline["traffic_note"] = "bytes per launch, scaled from the 256-table ncu capture in profiles/" if roofline["traffic"] else None
     t_alu = counts["fp64_slots"] / fma_rate
     t_hbm = counts["hbm_bytes"] / (hbm_gbs * 1e9)
     roofline["step"] = {"frac": max(t_alu, t_hbm) / step_s, "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
