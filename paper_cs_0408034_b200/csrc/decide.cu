@@ -34,8 +34,8 @@ __host__ __device__ inline size_t dec_layout(int npad, int nsp, unsigned char *b
 {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off += (bytes + 15) & ~size_t(15); return at; };
-    const size_t o_tab = take(3 * size_t(npad) * 8), o_gs = take(size_t(nsp) * 8), o_BC = take(size_t(nsp) * 16),
-                 o_Q = take(size_t(nsp) * 8), o_gm = take(kDecMG * 8), o_t = take(size_t(kDecMG) * kDecStride * 8),
+    const size_t o_tab = take(3 * size_t(npad) * 8), o_gs = take(size_t(nsp) * 8), o_BC = take(size_t(kDecMG) * nsp * 16),
+                 o_Q = take(size_t(kDecMG) * nsp * 8), o_gm = take(kDecMG * 8), o_t = take(size_t(kDecMG) * kDecStride * 8),
                  o_id = take(size_t(kDecMG) * (kDecTileP + 16)), o_si = take(size_t(kDecMG) * (kDecTileP + 16));
     if (o) {
         o->tab = reinterpret_cast<double *>(base + o_tab); o->gs = reinterpret_cast<double *>(base + o_gs);
@@ -83,6 +83,24 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     }
     const double g1 = gap_at(sm.tab, npad, 1.0);
     const double rdv = 2.0 * g1 + 3.0 * L;  // rendezvous handshake: 2 g(1) + 3 L
+    __syncthreads();
+    // line coefficients per (message size of the group, candidate): Section 2's k, Table 1's segmented rows
+    for (int idx = tid; idx < n_mi * nsp; idx += kDecThreads) {
+        const int mi = idx / nsp, si = idx - mi * nsp;
+        const uint32_t m_u = p.G.m_list[m0 + mi];
+        const int ns = p.G.ns_of_m[m0 + mi];
+        double B = CUDART_INF, C = CUDART_INF, Q = CUDART_INF;  // padding never wins
+        if (si < ns) {
+            const double gs = sm.gs[si];
+            const double k = static_cast<double>(segments(m_u, s_at(p.G, si), p.G.k_mode));
+            B = gs + L; C = gs * (k - 1.0); Q = gs * k;
+        } else if (ns == 0 && si == 0) {  // nothing fits: the whole message, k = 1
+            B = sm.gm[mi] + L; C = 0.0; Q = sm.gm[mi];
+        }
+        sm.cBC[idx] = make_double2(B, C);
+        sm.cQ[idx] = Q;
+    }
+    __syncthreads();
 
     // this thread's cells: process counts at tile offset warp*128 + r*32 + lane
     const int p_first = ptile * kDecTileP + warp * (32 * R) + lane;
@@ -100,6 +118,30 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     // the warp's pilot process count (middle of its range, clamped to the grid)
     const int P_mid = P_at(p.G, min(ptile * kDecTileP + warp * (32 * R) + 16 * R, p.G.n_P - 1));
     const double pm1_mid = static_cast<double>(P_mid - 1);
+
+    // Pilots for the whole group, issued together so that their latencies overlap: for each message size
+    // the chunk holding the candidate that is best at the warp's middle process count.  Only a guess that
+    // orders the work (float precision, candidate index in the low bits of the key); 4 bits per message size.
+    uint32_t pilotQ = 0, pilot5 = 0;
+    if (mask & ((1u << 2) | (1u << 5) | (1u << 9))) {
+#pragma unroll
+        for (int mi = 0; mi < kDecMG; ++mi) {
+            if (mi < n_mi) {
+                const int nsv = max(p.G.ns_of_m[m0 + mi], 1);
+                unsigned kq = 0xFFFFFFFFu, k5 = 0xFFFFFFFFu;
+                for (int c0 = 0; c0 < nsv; c0 += 32) {
+                    const int cand = c0 + lane;
+                    if (cand < nsv) {
+                        const double2 c = sm.cBC[mi * nsp + cand];
+                        kq = min(kq, (__float_as_uint(static_cast<float>(sm.cQ[mi * nsp + cand])) & ~63u) | static_cast<unsigned>(cand));
+                        k5 = min(k5, (__float_as_uint(static_cast<float>(fma(pm1_mid, c.x, c.y))) & ~63u) | static_cast<unsigned>(cand));
+                    }
+                }
+                pilotQ |= ((__reduce_min_sync(0xffffffffu, kq) & 63u) / U) << (4 * mi);
+                pilot5 |= ((__reduce_min_sync(0xffffffffu, k5) & 63u) / U) << (4 * mi);
+            }
+        }
+    }
 
     const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
 
@@ -124,26 +166,13 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     if (mask & 0x3FFu) {
         for (int mi = 0; mi < n_mi; ++mi) {
             const int midx = m0 + mi;
-            const uint32_t m_u = p.G.m_list[midx];
             const int ns = p.G.ns_of_m[midx];
             const int nsv = max(ns, 1);                 // candidates actually evaluated
             const int n_chunks = (nsv + U - 1) / U;
 
-            __syncthreads();  // the previous message size is done with the coefficient arrays
             const double gm = sm.gm[mi];
-            // line coefficients per candidate (Section 2's k, Table 1's segmented rows)
-            for (int si = tid; si < n_chunks * U; si += kDecThreads) {
-                double B = CUDART_INF, C = CUDART_INF, Q = CUDART_INF;  // padding never wins
-                if (si < ns) {
-                    const double gs = sm.gs[si];
-                    const double k = static_cast<double>(segments(m_u, s_at(p.G, si), p.G.k_mode));
-                    B = gs + L; C = gs * (k - 1.0); Q = gs * k;
-                } else if (ns == 0 && si == 0) {        // nothing fits: the whole message, k = 1
-                    B = gm + L; C = 0.0; Q = gm;
-                }
-                sm.cBC[si] = make_double2(B, C); sm.cQ[si] = Q;
-            }
-            __syncthreads();
+            const double2 *cBC = sm.cBC + mi * nsp;
+            const double *cQ = sm.cQ + mi * nsp;
 
             double bt[R];
             int bid[R];
@@ -156,20 +185,6 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                     if (val[r] < bt[r]) { bt[r] = val[r]; bid[r] = id; bsi[r] = sval ? sval[r] : kSiNone; }
             };
 
-            // Pilot: the candidate that is best for the process count in the middle of the warp's range.
-            // Only a guess that orders the work (float precision, index in the low bits of the key).
-            auto pilot_chunk = [&](auto eval_mid) {
-                unsigned key = 0xFFFFFFFFu;
-                for (int c0 = 0; c0 < nsv; c0 += 32) {
-                    const int cand = c0 + lane;
-                    if (cand < nsv) {
-                        const unsigned k = (__float_as_uint(static_cast<float>(eval_mid(cand))) & ~63u) | static_cast<unsigned>(cand);
-                        key = min(key, k);
-                    }
-                }
-                return static_cast<int>(__reduce_min_sync(0xffffffffu, key) & 63u) / U;
-            };
-            // Segmented model reduced over the candidates: eval(r, cand) is the model cell.
             // Segmented model reduced over the candidates: load(cand) fetches the candidate's line
             // coefficients from shared memory, eval(r, coef) is the model cell.
             auto segmented = [&](int id, int cp, auto load, auto eval) {
@@ -230,8 +245,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 consider(id, st, si);
             };
             // ids 2 and 9 are a_P * Q(s) + c_P with a_P > 0: their best candidate is the same for every P
-            int cpQ = 0;
-            if (mask & ((1u << 2) | (1u << 9))) cpQ = pilot_chunk([&](int cand) { return sm.cQ[cand]; });
+            const int cpQ = (pilotQ >> (4 * mi)) & 15;
 
             double v[R];
             if (mask & 1u) {  // Flat Tree
@@ -245,7 +259,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 consider(1, v, nullptr);
             }
             if ((mask >> 2) & 1u)  // Segmented Flat Tree
-                segmented(2, cpQ, [&](int cand) { return sm.cQ[cand]; }, [&](int r, double q) { return fma(pm1[r], q, L); });
+                segmented(2, cpQ, [&](int cand) { return cQ[cand]; }, [&](int r, double q) { return fma(pm1[r], q, L); });
             if ((mask >> 3) & 1u) {  // Chain
 #pragma unroll
                 for (int r = 0; r < R; ++r) v[r] = pm1[r] * (gm + L);
@@ -257,8 +271,8 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 consider(4, v, nullptr);
             }
             if ((mask >> 5) & 1u) {  // Segmented Chain
-                const int cp5 = pilot_chunk([&](int cand) { const double2 c = sm.cBC[cand]; return fma(pm1_mid, c.x, c.y); });
-                segmented(5, cp5, [&](int cand) { return sm.cBC[cand]; }, [&](int r, double2 c) { return fma(pm1[r], c.x, c.y); });
+                const int cp5 = (pilot5 >> (4 * mi)) & 15;
+                segmented(5, cp5, [&](int cand) { return cBC[cand]; }, [&](int r, double2 c) { return fma(pm1[r], c.x, c.y); });
             }
             if ((mask >> 6) & 1u) {  // Binary Tree (the printed bound)
 #pragma unroll
@@ -276,7 +290,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 consider(8, v, nullptr);
             }
             if ((mask >> 9) & 1u)  // Segmented Binomial Tree
-                segmented(9, cpQ, [&](int cand) { return sm.cQ[cand]; }, [&](int r, double q) { return fma(lf[r], q, lcL[r]); });
+                segmented(9, cpQ, [&](int cand) { return cQ[cand]; }, [&](int r, double q) { return fma(lf[r], q, lcL[r]); });
 
 #pragma unroll
             for (int r = 0; r < R; ++r) {
