@@ -186,3 +186,33 @@ def test_config3_full_size_sampled_cells(plogp):
             assert d_t[ip, im] <= time[other, ip, im] * (1 + 1e-9)
             assert int(np.uint32(d_s[ip, im])) == int(best[(2, 5).index(sid), ip, im])
     assert np.isnan(time[[0, 1, 3, 4, 6, 7, 8, 9, 10, 11, 12]]).all()
+
+
+def test_select_best_with_explicit_P_list_and_per_table_sizes(plogp):
+    """Decision kernels on a process-count list with gaps (Scatter Chain terms span several j) and on
+    tables that do not share their size lists."""
+    import torch
+    from oracle import plogp_oracle as po
+    rng_sizes = np.stack([wl.log_spaced_multiples(4, 1 << 20, 16), wl.log_spaced_multiples(8, 1 << 22, 16),
+                          wl.log_spaced_multiples(4, 1 << 18, 16)])
+    gaps = np.stack([wl.noisy_monotone_gaps(rng_sizes[t], 2.0 + t, 0.004 * (t + 1), 0.05, 77 + t) for t in range(3)])
+    lat = np.array([3.0, 11.0, 0.5])
+    P = np.array([2, 3, 5, 8, 13, 21, 34, 55, 89, 144, 233, 377, 610, 987], dtype=np.int32)
+    m = wl.log_spaced_multiples(4, 1 << 21, 21)
+    s = wl.log_spaced_multiples(4, 1 << 19, 11)
+    g = plogp.GridArgs(m, P=P, s=s)
+    with plogp.Tables(rng_sizes, gaps, lat) as tabs:
+        dec = plogp.select_best(tabs, g)
+        torch.cuda.synchronize()
+    sg = po.SGrid(s)
+    for t in range(3):
+        tab = po.Table(rng_sizes[t], gaps[t], lat[t])
+        od = po.select_grid(wl.ALL_STRATEGIES, po.predict_grid(tab, wl.ALL_STRATEGIES, P, m, sg))
+        got_id = dec.strategy[t].cpu().numpy()
+        got_s = dec.s_bytes[t].cpu().numpy().view(np.uint32)
+        got_t = dec.time[t].cpu().numpy()
+        margin = (od.runner_up - od.time) / od.time
+        clear = margin > 1e-9
+        assert (got_id[clear] == od.strategy[clear]).all() and (got_s[clear] == od.s[clear]).all()
+        assert np.max(np.abs(got_t - od.time) / od.time) <= 1e-9
+        assert np.max(np.abs(got_t[clear] - od.time[clear]) / od.time[clear]) <= 1e-12
