@@ -35,7 +35,13 @@ struct LineWalk {
     }
     __device__ __forceinline__ double at(const double *s_tab, int npad, double x)
     {
-        while (x >= next) { ++i; load(s_tab, npad); }
+        while (x >= next) {
+            // rare: keep it a branch (the barrier stops the compiler from turning the reload into
+            // loads and selects that would run at every step)
+            asm volatile("" ::: "memory");
+            ++i;
+            load(s_tab, npad);
+        }
         return fma(x - key, slope, gap);
     }
 };
@@ -43,7 +49,8 @@ struct LineWalk {
 }  // namespace
 
 // CONTIG: the process counts are the contiguous range P_lo + index (one new gap per step).
-template <bool CONTIG>
+// ALL: the three Scatter strategies are enabled (the usual case), known at compile time.
+template <bool CONTIG, bool ALL>
 __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -52,7 +59,7 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
     double *s_tot = s_cum + p.G.lc_max * 32;   // [kWarps][32]
     const int npad = p.T.npad;
     const uint32_t mask = p.G.mask;
-    const bool on10 = (mask >> 10) & 1u, on11 = (mask >> 11) & 1u, on12 = (mask >> 12) & 1u;
+    const bool on10 = ALL || ((mask >> 10) & 1u), on11 = ALL || ((mask >> 11) & 1u), on12 = ALL || ((mask >> 12) & 1u);
 
     int b = blockIdx.x;
     const int mtile = b % p.n_mtiles;
@@ -90,14 +97,20 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
     const int e0 = ptile * (kWarps * run_len) + warp * run_len;
     const int e1 = min(e0 + run_len, p.G.n_P);
 
-    // One step of the Chain sum: all gaps g(j m) with j from the previous process count (1 before
-    // the first) to P-1; a single gap when the process counts are contiguous.
-    auto chain_step = [&](int e, int P, LineWalk &w, double &x) -> double {
-        if (CONTIG && e > 0) {
-            const double g = w.at(s_tab, npad, x);
-            x += md;  // exact: j m < 2^53
-            return g;
+    // Chain sum.  Contiguous process counts: the step for index e is the single gap g((P-1) m), and the
+    // argument grows by m per step; only the very first index of the grid also owns the gaps below it
+    // (j = 1 .. P_lo - 2).  Listed process counts: the step owns all j from the previous count to P-1.
+    auto below_first = [&](LineWalk &w) {  // CONTIG, e0 == 0: sum of g(j m), j = 1 .. P_lo - 2
+        double sum = 0.0, comp = 0.0;
+        for (int j = 1; j <= p.G.P_lo - 2; ++j) {
+            const double y = w.at(s_tab, npad, static_cast<double>(j) * md) - comp;
+            const double t = sum + y;
+            comp = (t - sum) - y;
+            sum = t;
         }
+        return sum;
+    };
+    auto listed_step = [&](int e, int P, LineWalk &w) {  // !CONTIG
         const int jlo = e == 0 ? 1 : P_at(p.G, e - 1);
         double sum = 0.0, comp = 0.0;
         for (int j = jlo; j <= P - 1; ++j) {
@@ -106,22 +119,27 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
             comp = (t - sum) - y;
             sum = t;
         }
-        x = static_cast<double>(P) * md;
         return sum;
     };
-    auto first_arg = [&](int e) {  // smallest j m that the run starting at index e will look up
-        const int jlo = e == 0 ? 1 : P_at(p.G, e - 1);
-        return static_cast<double>(jlo) * md;
-    };
+    const int P0 = e0 < p.G.n_P ? P_at(p.G, e0) : 2;
+    const double x_first = static_cast<double>((e0 == 0 || !CONTIG) ? (e0 == 0 ? 1 : P_at(p.G, e0 - 1)) : P0 - 1) * md;
 
     double run = 0.0;
-    if (on11) {
+    if (on11) {  // first pass over the run, no stores: this warp's share of the sum
         double mine = 0.0;
         if (e0 < e1) {
             LineWalk w;
-            double x = first_arg(e0);
-            w.start(s_tab, npad, x);
-            for (int e = e0; e < e1; ++e) mine += chain_step(e, P_at(p.G, e), w, x);
+            w.start(s_tab, npad, x_first);
+            if (CONTIG) {
+                if (e0 == 0) mine = below_first(w);
+                double x = static_cast<double>(P0 - 1) * md;
+                for (int e = e0; e < e1; ++e) {
+                    mine += w.at(s_tab, npad, x);
+                    x += md;  // exact: j m < 2^53
+                }
+            } else {
+                for (int e = e0; e < e1; ++e) mine += listed_step(e, P_at(p.G, e), w);
+            }
         }
         s_tot[warp * 32 + lane] = mine;
     }
@@ -130,27 +148,32 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
         if (p.s1_carry) run = p.s1_carry[(static_cast<size_t>(trel) * p.n_ptiles + ptile) * p.G.n_m + midx_c];
         for (int w = 0; w < warp; ++w) run += s_tot[w * 32 + lane];
     }
-    if (e0 >= e1) return;
+    if (e0 >= e1 || !m_ok) return;  // no barriers below
 
     LineWalk w;
-    double x = first_arg(e0);
-    if (on11) w.start(s_tab, npad, x);
+    if (on11) {
+        w.start(s_tab, npad, x_first);
+        if (CONTIG && e0 == 0) run += below_first(w);
+    }
+    double x = static_cast<double>(P0 - 1) * md;
 
     const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
     size_t o = (static_cast<size_t>(table) * 2 + 1) * plane + static_cast<size_t>(e0) * p.G.n_m + midx;
-    int P = P_at(p.G, e0);
+    int P = P0;
     int lc = 32 - __clz(P - 1);               // ceil(log2 P)
+    int P_next_lc = (1 << lc) + 1;            // first process count with a larger ceil(log2 P)
     double lcL = static_cast<double>(lc) * L;
     double s2 = on12 ? s_cum[(lc - 1) * 32 + lane] + lcL : 0.0;
     double pm1 = static_cast<double>(P - 1);
 
     for (int e = e0; e < e1; ++e) {
-        if (!CONTIG || e == e0) {
+        if (!CONTIG) {
             P = P_at(p.G, e);
             pm1 = static_cast<double>(P - 1);
         }
-        if (32 - __clz(P - 1) != lc) {  // P passed a power of two
+        if (P >= P_next_lc) {  // P passed a power of two
             lc = 32 - __clz(P - 1);
+            P_next_lc = (1 << lc) + 1;
             lcL = static_cast<double>(lc) * L;
             if (on12) s2 = s_cum[(lc - 1) * 32 + lane] + lcL;
         }
@@ -158,19 +181,32 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
         int bid = 255;
         if (on10) { bt = fma(pm1, gm, L); bid = 10; }                    // Flat Tree
         if (on11) {                                                      // Chain
-            run += chain_step(e, P, w, x);
+            if (CONTIG) {
+                run += w.at(s_tab, npad, x);
+                x += md;
+            } else {
+                run += listed_step(e, P, w);
+            }
             const double t = fma(pm1, L, run);
             if (t < bt) { bt = t; bid = 11; }
         }
         if (on12 && s2 < bt) { bt = s2; bid = 12; }                      // Binomial Tree
-        if (m_ok) {
-            p.d_time[o] = bt;
-            p.d_strategy[o] = static_cast<uint8_t>(bid);
-            p.d_sbytes[o] = 0u;
-        }
+        p.d_time[o] = bt;
+        p.d_strategy[o] = static_cast<uint8_t>(bid);
+        p.d_sbytes[o] = 0u;
         o += p.G.n_m;
         if (CONTIG) { ++P; pm1 += 1.0; }
     }
+}
+
+template <bool CONTIG, bool ALL>
+static cudaError_t launch_scatter_t(const FusedParams &p, size_t smem, unsigned blocks, cudaStream_t st)
+{
+    cudaError_t e = cudaSuccess;
+    if (smem > 48 * 1024) e = cudaFuncSetAttribute(scatter_kernel<CONTIG, ALL>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    scatter_kernel<CONTIG, ALL><<<blocks, kThreads, smem, st>>>(p);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_scatter(const FusedParams &p, cudaStream_t st)
@@ -178,17 +214,10 @@ cudaError_t launch_scatter(const FusedParams &p, cudaStream_t st)
     const size_t smem = (3 * static_cast<size_t>(p.T.npad) + static_cast<size_t>(p.G.lc_max) * 32 + kWarps * 32) * sizeof(double);
     const long long blocks = static_cast<long long>(p.n_mtiles) * p.n_ptiles * p.n_tables_launch;
     if (blocks <= 0 || blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    cudaError_t e = cudaSuccess;
-    if (p.G.P_list == nullptr) {
-        if (smem > 48 * 1024) e = cudaFuncSetAttribute(scatter_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        if (e != cudaSuccess) return e;
-        scatter_kernel<true><<<static_cast<unsigned>(blocks), kThreads, smem, st>>>(p);
-    } else {
-        if (smem > 48 * 1024) e = cudaFuncSetAttribute(scatter_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        if (e != cudaSuccess) return e;
-        scatter_kernel<false><<<static_cast<unsigned>(blocks), kThreads, smem, st>>>(p);
-    }
-    return cudaGetLastError();
+    const unsigned nb = static_cast<unsigned>(blocks);
+    const bool all = (p.G.mask & 0x1C00u) == 0x1C00u, contig = p.G.P_list == nullptr;
+    if (contig) return all ? launch_scatter_t<true, true>(p, smem, nb, st) : launch_scatter_t<true, false>(p, smem, nb, st);
+    return all ? launch_scatter_t<false, true>(p, smem, nb, st) : launch_scatter_t<false, false>(p, smem, nb, st);
 }
 
 }  // namespace plogp
