@@ -57,7 +57,7 @@ def make_workload(name: str, scale: str, rank: int):
 
 
 def work_counts(w):
-    """Cells of one step and the algorithmic work of each kernel (DESIGN.md section 7): a segmented cell
+    """Cells of one step and the algorithmic work of each kernel: a segmented cell
     is one DFMA and one compare (2 FP64 issue slots), an unsegmented cell one DFMA, a Scatter Chain
     element one interpolation DFMA, one running-sum DADD and the model's DFMA; HBM bytes are the decision
     table written once (13 B per decision cell)."""
