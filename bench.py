@@ -295,17 +295,14 @@ def main():
     # ---- end to end through the public API with host buffers ----
     e2e_ms, h2d, d2h = None, 0, 0
     if args.e2e_steps > 0:
-        host = plogp.DecisionTable(*(torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (out.strategy, out.s_bytes, out.time)))
+        host = plogp.alloc_decision_host(w.n_tables, w.n_P, w.n_m)   # page-locked
         h2d = w.sizes.nbytes + w.gaps.nbytes + w.latency.nbytes + w.m.nbytes + (0 if w.s_list is None else w.s_list.nbytes)
         d2h = sum(t.numel() * t.element_size() for t in (host.strategy, host.s_bytes, host.time))
 
         def e2e_step():
-            with plogp.Tables.from_workload(w) as tb:   # host arrays -> device (inside plogp_table_load)
-                plogp.select_best(tb, grid, out=out)
-                host.strategy.copy_(out.strategy, non_blocking=True)
-                host.s_bytes.copy_(out.s_bytes, non_blocking=True)
-                host.time.copy_(out.time, non_blocking=True)
-                torch.cuda.synchronize()
+            # host arrays in (plogp_table_load), host arrays out (plogp_select_best_host): every copy is inside
+            with plogp.Tables.from_workload(w) as tb:
+                plogp.select_best_host(tb, grid, out=host)
 
         e2e_step()
         barrier()

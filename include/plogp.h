@@ -129,6 +129,19 @@ int plogp_predict(plogp_tables *tables, const plogp_grid *grid, double *d_time, 
 int plogp_select_best(plogp_tables *tables, const plogp_grid *grid, uint8_t *d_strategy,
                       uint32_t *d_s_bytes, double *d_time, void *stream);
 
+/*
+ * plogp_select_best with HOST outputs: the same decision table (Sections 1 and 5), delivered into the
+ * caller's host arrays h_strategy / h_s_bytes / h_time, each [n_tables][2][n_P][n_m].  The tables are
+ * processed in batches through two device staging sets owned by the handle (at most 512 MiB each, or one
+ * table), so the device never holds the whole decision table, and the device-to-host copy of one batch runs
+ * while the next batch is computed.  Page-locked host arrays are needed for that overlap (pageable ones work,
+ * more slowly).  Planes of a collective with no enabled strategy are copied from staging unchanged, i.e. their
+ * contents are unspecified.  The call returns after the last byte has arrived (it synchronises `stream` and
+ * its own copy stream); it may allocate staging memory on first use.
+ */
+int plogp_select_best_host(plogp_tables *tables, const plogp_grid *grid, uint8_t *h_strategy,
+                           uint32_t *h_s_bytes, double *h_time, void *stream);
+
 /* Static description of a status code. */
 const char *plogp_status_string(int status);
 

@@ -78,6 +78,11 @@ struct plogp_tables {
     size_t ws_cap = 0;
     Plan plan;
     // optional per-kernel timing: event pairs recorded around every launch while enabled
+    // host-output path: two device staging sets and a copy stream
+    unsigned char *d_stage[2] = {nullptr, nullptr};
+    size_t stage_cap = 0;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_done[2] = {nullptr, nullptr}, ev_copied[2] = {nullptr, nullptr};
     bool profiling = false;
     struct Timed { int kind; cudaEvent_t a, b; };
     std::vector<Timed> timed;
@@ -346,7 +351,7 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cudaStream_t st)
+int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cudaStream_t st, int t_begin = 0, int t_end = -1)
 {
     int dev = 0;
     CK(cudaGetDevice(&dev));
@@ -363,8 +368,9 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
     const int passes_per_tile = pl.passes_per_tile;
     const bool need_carry = s1 && n_ptiles > 1;
 
-    for (int t0 = 0; t0 < h->T.n_tables; t0 += pl.tables_per_batch) {
-        const int nt = std::min(pl.tables_per_batch, h->T.n_tables - t0);
+    if (t_end < 0) t_end = h->T.n_tables;
+    for (int t0 = t_begin; t0 < t_end; t0 += pl.tables_per_batch) {
+        const int nt = std::min(pl.tables_per_batch, t_end - t0);
         unsigned char *ws = h->d_ws;
         double *part_time = nullptr;
         uint32_t *part_idx = nullptr;
@@ -500,7 +506,12 @@ int plogp_table_free(plogp_tables *h)
 {
     if (!h) return PLOGP_OK;
     int rc = PLOGP_OK;
-    void *bufs[] = {h->d_tab, h->d_lat, h->d_grid, h->d_ws};
+    void *bufs[] = {h->d_tab, h->d_lat, h->d_grid, h->d_ws, h->d_stage[0], h->d_stage[1]};
+    for (int i = 0; i < 2; ++i) {
+        if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
+        if (h->ev_copied[i]) cudaEventDestroy(h->ev_copied[i]);
+    }
+    if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
     for (void *b : bufs) {
         if (b) {
             cudaError_t e = cudaFree(b);
@@ -555,6 +566,72 @@ int plogp_select_best(plogp_tables *tables, const plogp_grid *grid, uint8_t *d_s
     out.d_sbytes = d_s_bytes;
     out.d_time = d_time;
     return run(tables, grid, false, out, static_cast<cudaStream_t>(stream));
+}
+
+int plogp_select_best_host(plogp_tables *h, const plogp_grid *grid, uint8_t *h_strategy, uint32_t *h_s_bytes,
+                           double *h_time, void *stream)
+{
+    if (!h || !grid || !h_strategy || !h_s_bytes || !h_time) return PLOGP_E_INVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev != h->device) return PLOGP_E_INVAL;
+    int rc = prepare(h, grid, st);
+    if (rc != PLOGP_OK) { h->plan = Plan(); return rc; }
+    if (h->plan.empty) return PLOGP_OK;
+    const size_t cells = size_t(2) * h->plan.G.n_P * h->plan.G.n_m;  // per table
+    const size_t per_table = cells * 13 + 3 * 256;
+    // tables per staging set: at most 512 MiB, at least one table
+    const int batch = int(std::min<size_t>(h->T.n_tables, std::max<size_t>(1, (size_t(512) << 20) / per_table)));
+    const size_t need = per_table * batch;
+    if (need > h->stage_cap) {
+        for (int i = 0; i < 2; ++i) {
+            if (h->d_stage[i]) CK(cudaFree(h->d_stage[i]));
+            h->d_stage[i] = nullptr;
+        }
+        h->stage_cap = 0;
+        for (int i = 0; i < 2; ++i) {
+            cudaError_t e = cudaMalloc(&h->d_stage[i], need);
+            if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return PLOGP_E_NOMEM; }
+            if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(staging)");
+        }
+        h->stage_cap = need;
+    }
+    if (!h->copy_stream) {
+        CK(cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            CK(cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming));
+            CK(cudaEventCreateWithFlags(&h->ev_copied[i], cudaEventDisableTiming));
+        }
+    }
+    auto align = [](size_t x) { return (x + 255) / 256 * 256; };
+    int slot = 0;
+    for (int t0 = 0; t0 < h->T.n_tables; t0 += batch, slot ^= 1) {
+        const int nt = std::min(batch, h->T.n_tables - t0);
+        // layout of a staging set: time | segment size | strategy, each for nt tables
+        double *s_time = reinterpret_cast<double *>(h->d_stage[slot]);
+        uint32_t *s_sb = reinterpret_cast<uint32_t *>(h->d_stage[slot] + align(cells * 8 * batch));
+        uint8_t *s_id = h->d_stage[slot] + align(cells * 8 * batch) + align(cells * 4 * batch);
+        if (t0 >= 2 * batch) CK(cudaStreamWaitEvent(st, h->ev_copied[slot], 0));  // the set's previous copy has left
+        FusedParams out{};
+        // the kernels index outputs by absolute table number
+        out.d_time = s_time - size_t(t0) * cells;
+        out.d_sbytes = s_sb - size_t(t0) * cells;
+        out.d_strategy = s_id - size_t(t0) * cells;
+        rc = run(h, grid, false, out, st, t0, t0 + nt);
+        if (rc != PLOGP_OK) break;
+        CK(cudaEventRecord(h->ev_done[slot], st));
+        CK(cudaStreamWaitEvent(h->copy_stream, h->ev_done[slot], 0));
+        CK(cudaMemcpyAsync(h_time + size_t(t0) * cells, s_time, cells * 8 * nt, cudaMemcpyDeviceToHost, h->copy_stream));
+        CK(cudaMemcpyAsync(h_s_bytes + size_t(t0) * cells, s_sb, cells * 4 * nt, cudaMemcpyDeviceToHost, h->copy_stream));
+        CK(cudaMemcpyAsync(h_strategy + size_t(t0) * cells, s_id, cells * nt, cudaMemcpyDeviceToHost, h->copy_stream));
+        CK(cudaEventRecord(h->ev_copied[slot], h->copy_stream));
+    }
+    cudaError_t e1 = cudaStreamSynchronize(h->copy_stream), e2 = cudaStreamSynchronize(st);
+    if (rc != PLOGP_OK) return rc;
+    if (e1 != cudaSuccess) return cuda_fail(e1, "cudaStreamSynchronize(copy)");
+    if (e2 != cudaSuccess) return cuda_fail(e2, "cudaStreamSynchronize");
+    return PLOGP_OK;
 }
 
 const char *plogp_status_string(int status)

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libplogp.so")
 
 N_STRATEGIES = 13
 SEGMENTED_IDS = (2, 5, 9)
-EXPORTS = ("plogp_table_load", "plogp_table_free", "plogp_predict", "plogp_select_best",
+EXPORTS = ("plogp_table_load", "plogp_table_free", "plogp_predict", "plogp_select_best", "plogp_select_best_host",
            "plogp_status_string", "plogp_last_cuda_error", "plogp_kernel_launches", "plogp_fp64_fma_rate", "plogp_profile_enable", "plogp_profile_read",
            "plogp_scatter_chain_static")
 
@@ -51,6 +51,8 @@ lib.plogp_predict.restype = C.c_int
 lib.plogp_predict.argtypes = [C.c_void_p, C.POINTER(Grid), C.c_void_p, C.c_void_p, C.c_void_p]
 lib.plogp_select_best.restype = C.c_int
 lib.plogp_select_best.argtypes = [C.c_void_p, C.POINTER(Grid), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+lib.plogp_select_best_host.restype = C.c_int
+lib.plogp_select_best_host.argtypes = [C.c_void_p, C.POINTER(Grid), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.plogp_status_string.restype = C.c_char_p
 lib.plogp_status_string.argtypes = [C.c_int]
 lib.plogp_last_cuda_error.restype = C.c_char_p
@@ -268,3 +270,22 @@ def profile_read(tables: Tables) -> dict:
     n = (C.c_int32 * len(KERNEL_KINDS))()
     _check(lib.plogp_profile_read(tables.handle, ms, n), "plogp_profile_read")
     return {k: (ms[i], n[i]) for i, k in enumerate(KERNEL_KINDS) if n[i]}
+
+
+def alloc_decision_host(n_tables: int, n_P: int, n_m: int) -> DecisionTable:
+    """Page-locked host arrays shaped like a decision table (for ``select_best_host``)."""
+    import torch
+    shape = (n_tables, 2, n_P, n_m)
+    return DecisionTable(torch.empty(shape, dtype=torch.uint8, pin_memory=True),
+                         torch.empty(shape, dtype=torch.int32, pin_memory=True),
+                         torch.empty(shape, dtype=torch.float64, pin_memory=True))
+
+
+def select_best_host(tables: Tables, grid, out: Optional[DecisionTable] = None, stream=None) -> DecisionTable:
+    """``plogp_select_best_host``: the decision table delivered into host arrays (returns when complete)."""
+    g = _as_grid(grid)
+    if out is None:
+        out = alloc_decision_host(tables.n_tables, g.n_P, g.n_m)
+    _check(lib.plogp_select_best_host(tables.handle, g.ref, out.strategy.data_ptr(), out.s_bytes.data_ptr(),
+                                      out.time.data_ptr(), _stream_ptr(stream)), "plogp_select_best_host")
+    return out

@@ -216,3 +216,23 @@ def test_select_best_with_explicit_P_list_and_per_table_sizes(plogp):
         assert (got_id[clear] == od.strategy[clear]).all() and (got_s[clear] == od.s[clear]).all()
         assert np.max(np.abs(got_t - od.time) / od.time) <= 1e-9
         assert np.max(np.abs(got_t[clear] - od.time[clear]) / od.time[clear]) <= 1e-12
+
+
+def test_host_output_entry_point_matches_device_outputs(plogp):
+    """plogp_select_best_host streams the decision table to host arrays in batches (here 3 batches of
+    tables through the two staging sets); it must equal plogp_select_best bit for bit."""
+    import torch
+    w = wl.config4(n_tables=700)
+    with plogp.Tables.from_workload(w) as tabs:
+        dev = plogp.select_best(tabs, w)
+        host = plogp.select_best_host(tabs, w)
+        host2 = plogp.select_best_host(tabs, w)   # staging sets and events are reused
+        torch.cuda.synchronize()
+    for h in (host, host2):
+        assert torch.equal(h.strategy, dev.strategy.cpu())
+        assert torch.equal(h.s_bytes, dev.s_bytes.cpu())
+        assert torch.equal(h.time.view(torch.int64), dev.time.cpu().view(torch.int64))
+    small = wl.config1()
+    with plogp.Tables.from_workload(small) as tabs:
+        a, b = plogp.select_best(tabs, small), plogp.select_best_host(tabs, small)
+    assert torch.equal(b.strategy, a.strategy.cpu()) and torch.equal(b.time.view(torch.int64), a.time.cpu().view(torch.int64))
