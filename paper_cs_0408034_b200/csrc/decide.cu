@@ -1,6 +1,6 @@
 // decide_kernel: Broadcast half of the decision table (Sections 1 and 5 of the paper) for short
 // candidate lists, with lanes mapped to the process count P.  (The Scatter half has no candidate
-// lists and goes through fused_kernel.)
+// lists and goes through scatter_kernel.)
 //
 // One CTA owns one table, a group of 8 message sizes and a tile of 512 process counts (4 warps x
 // 32 lanes x 4 cells).  For a fixed (m, s) the segmented models of Table 1 are lines in P, so the
@@ -10,7 +10,7 @@
 // so a smaller double never has a larger high word); only chunks of candidates in which some cell
 // can improve run the exact FP64 compare-and-select pass.  To make that pass rare, each warp first
 // finds the best candidate for the process count in the middle of its range (one candidate per
-// lane, shuffle argmin) and evaluates that candidate's chunk first: neighbouring process counts
+// lane, one warp-wide integer minimum over float keys) and evaluates that candidate's chunk first: neighbouring process counts
 // nearly always share the optimum, and for ids 2 and 9 the optimum does not depend on P at all.
 //
 // Results are staged in shared memory as [m][P] and written out as rows of 8 consecutive m.

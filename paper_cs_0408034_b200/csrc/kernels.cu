@@ -2,15 +2,19 @@
 // of "Fast Tuning of Intra-Cluster Collective Communications", the segment-size search of
 // Section 3.1 and the strategy selection of Sections 1 and 5.
 //
-// Two kernel families:
+// This file:
 //   sweep_kernel   lane <-> process count P.  One CTA owns one message size m, a tile of P values
 //                  and a chunk of the candidate segment sizes; the per-(m, s) line coefficients are
 //                  computed once per CTA into shared memory and broadcast to all lanes, so a model
-//                  cell costs one DFMA and one compare.  Used when the candidate list is long.
+//                  cell costs one DFMA and one integer compare.  Used when the candidate list is long.
 //   fused_kernel   lane <-> message size m (32 consecutive m per warp, so every output row is
 //                  written as full, aligned segments).  Evaluates all enabled strategies, runs short
-//                  candidate lists inline, block-scans the Scatter Chain sum over P, and writes
-//                  either the predicted planes or the decision table.
+//                  candidate lists inline or reduces the sweep kernel's partial minima, keeps the
+//                  Scatter Chain sum running along each warp's contiguous run of P, and writes either
+//                  the predicted planes or the decision table.  The general path.
+//   s1_tile_*      tile sums and their scan for the Scatter Chain sum when P is split over CTAs.
+// The decision table of short candidate lists has faster, specialised kernels in decide.cu
+// (Broadcast half) and scatter.cu (Scatter half).
 #include "device_common.cuh"
 
 namespace plogp {
