@@ -412,16 +412,17 @@ __global__ void __launch_bounds__(kThreads) fused_kernel(const FusedParams p)
             }
         };
         auto flush = [&](int coll) {
-            if (PREDICT) return;
+            if constexpr (!PREDICT) {
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                if (ok[r] && m_ok) {
-                    const size_t o = out_index(coll, 2, r);
-                    p.d_strategy[o] = static_cast<uint8_t>(bid[r]);
-                    p.d_sbytes[o] = bsz[r];
-                    p.d_time[o] = bt[r];
+                for (int r = 0; r < R; ++r) {
+                    if (ok[r] && m_ok) {
+                        const size_t o = out_index(coll, 2, r);
+                        p.d_strategy[o] = static_cast<uint8_t>(bid[r]);
+                        p.d_sbytes[o] = bsz[r];
+                        p.d_time[o] = bt[r];
+                    }
+                    bt[r] = CUDART_INF; bsz[r] = 0; bid[r] = 255;
                 }
-                bt[r] = CUDART_INF; bsz[r] = 0; bid[r] = 255;
             }
         };
 

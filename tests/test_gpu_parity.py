@@ -236,3 +236,12 @@ def test_host_output_entry_point_matches_device_outputs(plogp):
     with plogp.Tables.from_workload(small) as tabs:
         a, b = plogp.select_best(tabs, small), plogp.select_best_host(tabs, small)
     assert torch.equal(b.strategy, a.strategy.cpu()) and torch.equal(b.time.view(torch.int64), a.time.cpu().view(torch.int64))
+
+
+def test_sweep_kernel_with_several_tables(plogp):
+    """Long candidate list (512 multiples of 4 B) on three independent tables: the sweep kernel's table
+    dimension and the reduction of its partial minima per table."""
+    from dataclasses import replace
+    base = wl.config4(n_tables=3, P_hi=70, n_m=9)
+    w = replace(base, s_list=None, s_lo=4, s_hi=2048, s_step=4)
+    run_both(plogp, w)
