@@ -47,3 +47,34 @@ def test_grid_struct_matches_the_header_layout(tmp_path):
     got = [int(x) for x in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
     assert got[0] == ctypes.sizeof(plogp.Grid)
     assert got[1:] == [getattr(plogp.Grid, f).offset for f in fields]
+
+
+def test_table_validation_runs_on_the_host_before_any_device_call():
+    """Malformed tables are refused with a status code without touching CUDA (works without a GPU)."""
+    import numpy as np
+    from paper_cs_0408034_b200 import plogp
+
+    def status(sizes, gaps, lat, shared=1):
+        sizes = np.ascontiguousarray(sizes, dtype=np.uint64)
+        gaps = np.ascontiguousarray(gaps, dtype=np.float64)
+        lat = np.ascontiguousarray(lat, dtype=np.float64)
+        h = ctypes.c_void_p()
+        rc = plogp.lib.plogp_table_load(gaps.shape[0], gaps.shape[1], sizes.ctypes.data, shared, gaps.ctypes.data,
+                                        lat.ctypes.data, ctypes.byref(h))
+        assert h.value is None or rc == 0
+        if rc == 0:
+            plogp.lib.plogp_table_free(h)
+        return rc
+
+    assert status([4, 4, 16], [[1.0, 2.0, 3.0]], [1.0]) == plogp.E_INVAL
+    assert status([4, 8, 16], [[1.0, float("nan"), 3.0]], [1.0]) == plogp.E_INVAL
+    assert status([4, 8, 16], [[1.0, 2.0, 3.0]], [-1.0]) == plogp.E_INVAL
+    assert status([4], [[1.0]], [1.0]) == plogp.E_INVAL
+    assert status([4, 8, 1 << 60], [[1.0, 2.0, 3.0]], [1.0]) == plogp.E_RANGE
+    assert status([[4, 8, 16], [4, 8, 8]], [[1.0, 2.0, 3.0], [1.0, 2.0, 3.0]], [1.0, 1.0], shared=0) == plogp.E_INVAL
+    h = ctypes.c_void_p()
+    assert plogp.lib.plogp_table_load(1, 3, None, 1, None, None, ctypes.byref(h)) == plogp.E_INVAL
+    assert plogp.lib.plogp_select_best(None, None, None, None, None, None) == plogp.E_INVAL
+    assert plogp.lib.plogp_predict(None, None, None, None, None) == plogp.E_INVAL
+    assert plogp.lib.plogp_scatter_chain_static(8, None, None, 1.0, 2, 3, None, 1, None, None) == plogp.E_INVAL
+    assert plogp.lib.plogp_table_free(None) == plogp.OK
