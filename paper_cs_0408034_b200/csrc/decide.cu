@@ -175,14 +175,13 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             const double *cQ = sm.cQ + mi * nsp;
 
             double bt[R];
-            int bid[R];
-            uint32_t bsi[R];
+            uint32_t bcode[R];  // winner so far: strategy id << 8 | candidate index (or kSiNone / kSiWhole)
 #pragma unroll
-            for (int r = 0; r < R; ++r) { bt[r] = CUDART_INF; bid[r] = 255; bsi[r] = kSiNone; }
+            for (int r = 0; r < R; ++r) { bt[r] = CUDART_INF; bcode[r] = (255u << 8) | kSiNone; }
             auto consider = [&](int id, const double *val, const uint32_t *sval) {
 #pragma unroll
                 for (int r = 0; r < R; ++r)
-                    if (val[r] < bt[r]) { bt[r] = val[r]; bid[r] = id; bsi[r] = sval ? sval[r] : kSiNone; }
+                    if (val[r] < bt[r]) { bt[r] = val[r]; bcode[r] = (static_cast<uint32_t>(id) << 8) | (sval ? sval[r] : kSiNone); }
             };
 
             // Segmented model reduced over the candidates: load(cand) fetches the candidate's line
@@ -296,8 +295,8 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             for (int r = 0; r < R; ++r) {
                 const int pr = warp * (32 * R) + 32 * r + lane;
                 sm.st_time[mi * kDecStride + pr] = bt[r];
-                sm.st_id[mi * (kDecTileP + 16) + pr] = static_cast<uint8_t>(bid[r]);
-                sm.st_si[mi * (kDecTileP + 16) + pr] = static_cast<uint8_t>(bsi[r]);
+                sm.st_id[mi * (kDecTileP + 16) + pr] = static_cast<uint8_t>(bcode[r] >> 8);
+                sm.st_si[mi * (kDecTileP + 16) + pr] = static_cast<uint8_t>(bcode[r] & 255u);
             }
         }
         __syncthreads();
