@@ -245,3 +245,31 @@ def test_sweep_kernel_with_several_tables(plogp):
     base = wl.config4(n_tables=3, P_hi=70, n_m=9)
     w = replace(base, s_list=None, s_lo=4, s_hi=2048, s_step=4)
     run_both(plogp, w)
+
+
+def test_exact_ties_go_to_smallest_segment_and_lowest_id(plogp):
+    """A flat table (g = 1 everywhere, L = 2) makes every model an exact small integer, so ties between
+    candidates with the same segment count and between strategies are exact on both sides: the GPU must
+    then reproduce the oracle's picks bit for bit (smallest s, lowest id), whatever order it sweeps in."""
+    import torch
+    from oracle import plogp_oracle as po
+    sizes = np.array([4, 64, 1024, 1 << 20], dtype=np.uint64)
+    gaps = np.ones((1, 4))
+    lat = np.array([2.0])
+    m = np.array([8, 100, 1000, 4096, 10000, 65536, 100000], dtype=np.uint64)
+    P = np.arange(2, 140, dtype=np.int32)
+    tab = po.Table(sizes, gaps[0], 2.0)
+    for s_kw, sg in ((dict(s=wl.log_spaced_multiples(4, 1 << 16, 40)), po.SGrid(wl.log_spaced_multiples(4, 1 << 16, 40))),
+                     (dict(s=None, s_lo=4, s_hi=4096, s_step=4), po.SGrid(lo=4, hi=4096, step=4))):
+        g = plogp.GridArgs(m, P=P, **s_kw)
+        with plogp.Tables(sizes, gaps, lat) as tabs:
+            dec = plogp.select_best(tabs, g)
+            pred = plogp.predict(tabs, g)
+            torch.cuda.synchronize()
+        o = po.predict_grid(tab, wl.ALL_STRATEGIES, P, m, sg)
+        od = po.select_grid(wl.ALL_STRATEGIES, o)
+        assert np.array_equal(pred.time[0].cpu().numpy(), o.time)
+        assert np.array_equal(pred.best_s[0].cpu().numpy().view(np.uint32), o.best_s)
+        assert np.array_equal(dec.strategy[0].cpu().numpy(), od.strategy)
+        assert np.array_equal(dec.s_bytes[0].cpu().numpy().view(np.uint32), od.s)
+        assert np.array_equal(dec.time[0].cpu().numpy(), od.time)
