@@ -233,18 +233,37 @@ __global__ void __launch_bounds__(kThreads) s1_tile_sum_kernel(const S1Params p)
     }
 }
 
-// Exclusive scan of the tile sums along the tile index, in place (one thread per (table, m)).
+// Exclusive scan of the tile sums along the tile index, in place: one warp per (table, m), each lane a
+// contiguous block of at most kScanPerLane tiles (n_ptiles <= 32 * kScanPerLane = 256).
+constexpr int kScanPerLane = 8;
 __global__ void s1_tile_scan_kernel(double *tile_sum, int n_tables, int n_ptiles, int n_m)
 {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n_tables * n_m) return;
+    const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (i >= n_tables * n_m) return;  // whole warps leave together
     const int trel = i / n_m, midx = i - trel * n_m;
-    double run = 0.0;
-    for (int pt = 0; pt < n_ptiles; ++pt) {
-        double *q = tile_sum + (static_cast<size_t>(trel) * n_ptiles + pt) * n_m + midx;
-        const double v = *q;
-        *q = run;
-        run += v;
+    const int per = (n_ptiles + 31) / 32;
+    double *base = tile_sum + static_cast<size_t>(trel) * n_ptiles * n_m + midx;
+    double v[kScanPerLane];
+    double mine = 0.0;
+#pragma unroll
+    for (int k = 0; k < kScanPerLane; ++k) {
+        const int pt = lane * per + k;
+        v[k] = (k < per && pt < n_ptiles) ? base[static_cast<size_t>(pt) * n_m] : 0.0;
+        mine += v[k];
+    }
+    double incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const double y = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += y;
+    }
+    double run = __shfl_up_sync(0xffffffffu, incl, 1);  // sum of the lower lanes' blocks
+    if (lane == 0) run = 0.0;
+#pragma unroll
+    for (int k = 0; k < kScanPerLane; ++k) {
+        const int pt = lane * per + k;
+        if (k < per && pt < n_ptiles) base[static_cast<size_t>(pt) * n_m] = run;
+        run += v[k];
     }
 }
 
@@ -641,7 +660,8 @@ cudaError_t launch_s1_tiles(const S1Params &p, cudaStream_t st)
     s1_tile_sum_kernel<<<static_cast<unsigned>(blocks), kThreads, smem, st>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const int n = p.n_tables_launch * p.G.n_m;
-    s1_tile_scan_kernel<<<(n + 127) / 128, 128, 0, st>>>(p.tile_sum, p.n_tables_launch, p.n_ptiles, p.G.n_m);
+    if (p.n_ptiles > 32 * kScanPerLane) return cudaErrorInvalidConfiguration;  // the host plan caps the tile count at 256
+    s1_tile_scan_kernel<<<(n + 3) / 4, 128, 0, st>>>(p.tile_sum, p.n_tables_launch, p.n_ptiles, p.G.n_m);
     return cudaGetLastError();
 }
 
