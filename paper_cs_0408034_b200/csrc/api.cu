@@ -56,7 +56,7 @@ struct Plan {
     // fused kernel tiling
     int n_mtiles = 0, n_ptiles = 1, passes_per_tile = 1;
     // decision kernel tiling (short candidate lists)
-    int dec_mgroups = 0, dec_ptiles = 1;
+    int dec_mgroups = 0, dec_ptiles = 1, dec_mg = kDecMG;
     size_t carry_bytes_per_table = 0;
     // sweep kernel
     int n_pairs = 0, sweep_ptiles = 0, chunk_len = 0;
@@ -259,8 +259,12 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     pl.passes_per_tile = (total_passes + n_ptiles - 1) / n_ptiles;
     pl.n_ptiles = (total_passes + pl.passes_per_tile - 1) / pl.passes_per_tile;
 
-    pl.dec_mgroups = (n_m + kDecMG - 1) / kDecMG;
     pl.dec_ptiles = (n_P + kDecTileP - 1) / kDecTileP;
+    // 8 message sizes per CTA give the widest output rows; small grids trade that for more CTAs
+    pl.dec_mg = kDecMG;
+    while (pl.dec_mg > 1 && (long long)((n_m + pl.dec_mg - 1) / pl.dec_mg) * pl.dec_ptiles * h->T.n_tables < (long long)h->sm_count * 4)
+        pl.dec_mg >>= 1;
+    pl.dec_mgroups = (n_m + pl.dec_mg - 1) / pl.dec_mg;
 
     // ---- device arrays ----
     std::vector<unsigned char> blob;
@@ -409,7 +413,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             DecideParams dp{};
             dp.T = h->T; dp.G = pl.G;
             dp.G.mask &= 0x3FFu;
-            dp.n_mgroups = pl.dec_mgroups; dp.n_ptiles = pl.dec_ptiles;
+            dp.n_mgroups = pl.dec_mgroups; dp.n_ptiles = pl.dec_ptiles; dp.mg = pl.dec_mg;
             dp.table0 = t0; dp.n_tables_launch = nt;
             dp.d_strategy = out.d_strategy; dp.d_sbytes = out.d_sbytes; dp.d_time = out.d_time;
             { LaunchTimer lt(h, PLOGP_KERNEL_DECIDE, st); CK(launch_decide(dp, st)); }

@@ -69,8 +69,8 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     const int trel = b / p.n_ptiles;
     const int table = p.table0 + trel;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int m0 = mgroup * kDecMG;
-    const int n_mi = min(kDecMG, p.G.n_m - m0);
+    const int m0 = mgroup * p.mg;   // p.mg <= kDecMG message sizes per CTA (fewer on small grids, for more CTAs)
+    const int n_mi = min(p.mg, p.G.n_m - m0);
 
     stage_table(sm.tab, p.T, table);
     __syncthreads();

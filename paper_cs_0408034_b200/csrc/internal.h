@@ -81,6 +81,7 @@ struct DecideParams {
     TableDev T;
     GridDev G;
     int n_mgroups, n_ptiles;
+    int mg;  // message sizes per CTA, 1..kDecMG
     int table0, n_tables_launch;
     uint8_t *d_strategy;
     uint32_t *d_sbytes;
@@ -91,7 +92,7 @@ constexpr int kDecThreads = 128;
 constexpr int kDecWarps = kDecThreads / 32;
 constexpr int kDecR = 4;                               // process counts per thread
 constexpr int kDecTileP = kDecThreads * kDecR;         // 512 process counts per CTA
-constexpr int kDecMG = 8;                              // message sizes per CTA
+constexpr int kDecMG = 8;                              // message sizes per CTA (at most)
 constexpr int kDecU = 4;                               // candidates per filter test
 
 constexpr int kThreads = 256;
