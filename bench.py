@@ -300,9 +300,9 @@ def main():
         d2h = sum(t.numel() * t.element_size() for t in (host.strategy, host.s_bytes, host.time))
 
         def e2e_step():
-            # host arrays in (plogp_table_load), host arrays out (plogp_select_best_host): every copy is inside
-            with plogp.Tables.from_workload(w) as tb:
-                plogp.select_best_host(tb, grid, out=host)
+            # host arrays in (plogp_table_update), host arrays out (plogp_select_best_host): every copy is inside
+            tabs.update(w.sizes, w.gaps, w.latency)
+            plogp.select_best_host(tabs, grid, out=host)
 
         e2e_step()
         barrier()

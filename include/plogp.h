@@ -80,6 +80,16 @@ typedef struct plogp_tables plogp_tables;
 int plogp_table_load(int n_tables, int n_bp, const uint64_t *sizes_bytes, int sizes_shared,
                      const double *gap, const double *latency, plogp_tables **out);
 
+/*
+ * Replace the contents of every table of a handle (same n_tables and n_bp as at plogp_table_load; same
+ * argument meaning and checks) without reallocating anything: for callers that re-tune the same grid as the
+ * measured pLogP parameters of Section 2 change.  The host arrays are copied before the call returns; the
+ * device copy is enqueued on `stream`, ordered before later calls on that stream.  On an error the tables on the
+ * device are unchanged.
+ */
+int plogp_table_update(plogp_tables *tables, const uint64_t *sizes_bytes, int sizes_shared,
+                       const double *gap, const double *latency, void *stream);
+
 /* Release a handle and its device memory (synchronises). NULL is accepted. */
 int plogp_table_free(plogp_tables *tables);
 

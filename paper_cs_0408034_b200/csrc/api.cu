@@ -443,16 +443,10 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
 
 extern "C" {
 
-int plogp_table_load(int n_tables, int n_bp, const uint64_t *sizes_bytes, int sizes_shared,
-                     const double *gap, const double *latency, plogp_tables **out)
+// Validates host tables and lays them out as the kernels read them (key | gap | slope, padded).
+static int build_tables(int n_tables, int n_bp, int npad, const uint64_t *sizes_bytes, int sizes_shared,
+                        const double *gap, const double *latency, std::vector<double> &tab, std::vector<double> &lat)
 {
-    if (!sizes_bytes || !gap || !latency || !out) return PLOGP_E_INVAL;
-    if (n_tables < 1 || n_bp < 2) return PLOGP_E_INVAL;
-    if (n_bp > PLOGP_MAX_BREAKPOINTS) return PLOGP_E_RANGE;
-    int npad = 2;
-    while (npad < n_bp) npad <<= 1;  // >= n_bp: at least one +inf key follows the last interval
-
-    std::vector<double> tab, lat;
     try {
         tab.assign(size_t(n_tables) * 3 * npad, 0.0);
         lat.assign(latency, latency + n_tables);
@@ -481,6 +475,21 @@ int plogp_table_load(int n_tables, int n_bp, const uint64_t *sizes_bytes, int si
             }
         }
     }
+    return PLOGP_OK;
+}
+
+int plogp_table_load(int n_tables, int n_bp, const uint64_t *sizes_bytes, int sizes_shared,
+                     const double *gap, const double *latency, plogp_tables **out)
+{
+    if (!sizes_bytes || !gap || !latency || !out) return PLOGP_E_INVAL;
+    if (n_tables < 1 || n_bp < 2) return PLOGP_E_INVAL;
+    if (n_bp > PLOGP_MAX_BREAKPOINTS) return PLOGP_E_RANGE;
+    int npad = 2;
+    while (npad < n_bp) npad <<= 1;  // >= n_bp: at least one +inf key follows the last interval
+
+    std::vector<double> tab, lat;
+    const int brc = build_tables(n_tables, n_bp, npad, sizes_bytes, sizes_shared, gap, latency, tab, lat);
+    if (brc != PLOGP_OK) return brc;
 
     plogp_tables *h = new (std::nothrow) plogp_tables();
     if (!h) return PLOGP_E_NOMEM;
@@ -503,6 +512,23 @@ int plogp_table_load(int n_tables, int n_bp, const uint64_t *sizes_bytes, int si
     h->T.n_bp = n_bp;
     h->T.npad = npad;
     *out = h;
+    return PLOGP_OK;
+}
+
+int plogp_table_update(plogp_tables *h, const uint64_t *sizes_bytes, int sizes_shared, const double *gap,
+                       const double *latency, void *stream)
+{
+    if (!h || !sizes_bytes || !gap || !latency) return PLOGP_E_INVAL;
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev != h->device) return PLOGP_E_INVAL;
+    std::vector<double> tab, lat;
+    const int brc = build_tables(h->T.n_tables, h->T.n_bp, h->T.npad, sizes_bytes, sizes_shared, gap, latency, tab, lat);
+    if (brc != PLOGP_OK) return brc;  // the tables on the device are untouched
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // pageable sources: the runtime stages them before returning, so the vectors may go out of scope
+    CK(cudaMemcpyAsync(h->d_tab, tab.data(), tab.size() * sizeof(double), cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(h->d_lat, lat.data(), lat.size() * sizeof(double), cudaMemcpyHostToDevice, st));
     return PLOGP_OK;
 }
 

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libplogp.so")
 
 N_STRATEGIES = 13
 SEGMENTED_IDS = (2, 5, 9)
-EXPORTS = ("plogp_table_load", "plogp_table_free", "plogp_predict", "plogp_select_best", "plogp_select_best_host",
+EXPORTS = ("plogp_table_load", "plogp_table_update", "plogp_table_free", "plogp_predict", "plogp_select_best", "plogp_select_best_host",
            "plogp_status_string", "plogp_last_cuda_error", "plogp_kernel_launches", "plogp_fp64_fma_rate", "plogp_profile_enable", "plogp_profile_read",
            "plogp_scatter_chain_static")
 
@@ -45,6 +45,8 @@ for _name in EXPORTS:
 lib.plogp_table_load.restype = C.c_int
 lib.plogp_table_load.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
                                  C.POINTER(C.c_void_p)]
+lib.plogp_table_update.restype = C.c_int
+lib.plogp_table_update.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.plogp_table_free.restype = C.c_int
 lib.plogp_table_free.argtypes = [C.c_void_p]
 lib.plogp_predict.restype = C.c_int
@@ -109,6 +111,18 @@ class Tables:
     @classmethod
     def from_workload(cls, w) -> "Tables":
         return cls(w.sizes, w.gaps, w.latency)
+
+    def update(self, sizes, gaps, latency, stream=None) -> None:
+        """``plogp_table_update``: new contents for all tables (same shapes), no reallocation."""
+        sizes = np.ascontiguousarray(sizes, dtype=np.uint64)
+        gaps = np.ascontiguousarray(gaps, dtype=np.float64)
+        latency = np.ascontiguousarray(latency, dtype=np.float64)
+        if gaps.shape != (self.n_tables, self.n_bp) or latency.shape != (self.n_tables,):
+            raise ValueError("shapes must match the loaded tables")
+        if sizes.shape != (self.n_bp,) and sizes.shape != gaps.shape:
+            raise ValueError("sizes must be [n_bp] or [n_tables][n_bp]")
+        _check(lib.plogp_table_update(self.handle, _ptr(sizes), int(sizes.ndim == 1), _ptr(gaps), _ptr(latency),
+                                      _stream_ptr(stream)), "plogp_table_update")
 
     @property
     def handle(self):

@@ -273,3 +273,22 @@ def test_exact_ties_go_to_smallest_segment_and_lowest_id(plogp):
         assert np.array_equal(dec.strategy[0].cpu().numpy(), od.strategy)
         assert np.array_equal(dec.s_bytes[0].cpu().numpy().view(np.uint32), od.s)
         assert np.array_equal(dec.time[0].cpu().numpy(), od.time)
+
+
+def test_table_update_replaces_contents_in_place(plogp):
+    import torch
+    a, b = wl.config4(n_tables=5, P_hi=40, n_m=12), wl.config4(n_tables=5, P_hi=40, n_m=12, seed_offset=9)
+    with plogp.Tables.from_workload(a) as tabs:
+        first = plogp.select_best(tabs, a)
+        tabs.update(b.sizes, b.gaps, b.latency)
+        second = plogp.select_best(tabs, b)
+        torch.cuda.synchronize()
+        check_decision(b, oracle_tables(b), second)
+        assert not torch.equal(first.time, second.time)
+        bad = b.gaps.copy()
+        bad[2, 3] = float("nan")
+        with pytest.raises(plogp.PlogpError):
+            tabs.update(b.sizes, bad, b.latency)
+        again = plogp.select_best(tabs, b)       # device tables untouched by the refused update
+        torch.cuda.synchronize()
+        assert torch.equal(again.time.view(torch.int64), second.time.view(torch.int64))
