@@ -214,8 +214,8 @@ int plogp_profile_read(plogp_tables *tables, double *ms, int32_t *launches);
 uint64_t plogp_kernel_launches(void);
 
 /*
- * Measurement aid with no counterpart in the paper: runs a register-only chain-free stream of
- * double-precision fused multiply-adds on every SM of the current device for about
+ * Measurement aid with no counterpart in the paper: runs a register-only stream of double-precision
+ * fused multiply-adds (16 independent chains per thread) on every SM of the current device for about
  * `milliseconds` and returns the sustained rate in thread-level FMA instructions per second
  * (the issue ceiling the segment sweep is compared with).  Synchronises.  Negative on error.
  */

@@ -689,7 +689,7 @@ double plogp_fp64_fma_rate(double milliseconds)
     double *sink = nullptr;
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     double rate = double(PLOGP_E_CUDA);
-    const int blocks = sms * 8;
+    const int blocks = sms * 4;
     const double fma_per_iter = double(blocks) * kThreads * 32.0;
     do {
         if (cudaMalloc(&sink, sizeof(double)) != cudaSuccess) break;
