@@ -243,6 +243,69 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 }
                 consider(id, st, si);
             };
+            // Ids 2 and 9 together: both read Q(s), so one sweep loads it once and tests 32 cells per branch.
+            double st9[R];
+            uint32_t si9[R];
+            auto segmented_2_and_9 = [&](int cp) {
+                double st2[R];
+                uint32_t si2[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) { st2[r] = st9[r] = CUDART_INF; si2[r] = si9[r] = 0; }
+#pragma unroll 1
+                for (int u = 0; u < U; ++u) {  // the pilot's chunk first, ascending, strict '<'
+                    const uint32_t cand = cp * U + u;
+                    const double q = cQ[cand];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const double t2 = fma(pm1[r], q, L), t9 = fma(lf[r], q, lcL[r]);
+                        if (t2 < st2[r]) { st2[r] = t2; si2[r] = cand; }
+                        if (t9 < st9[r]) { st9[r] = t9; si9[r] = cand; }
+                    }
+                }
+                double cur[U], nxt[U];
+                int chunk = cp == 0 ? 1 : 0;
+#pragma unroll
+                for (int u = 0; u < U; ++u) cur[u] = cQ[min(chunk, n_chunks - 1) * U + u];
+                while (chunk < n_chunks) {
+                    int next = chunk + 1;
+                    next += next == cp;
+#pragma unroll
+                    for (int u = 0; u < U; ++u) nxt[u] = cQ[min(next, n_chunks - 1) * U + u];
+                    bool f2[R], f9[R];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) f2[r] = f9[r] = false;
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            f2[r] |= __double2hiint(fma(pm1[r], cur[u], L)) <= __double2hiint(st2[r]);
+                            f9[r] |= __double2hiint(fma(lf[r], cur[u], lcL[r])) <= __double2hiint(st9[r]);
+                        }
+                    }
+                    const bool a2 = (f2[0] | f2[1]) | (f2[2] | f2[3]), a9 = (f9[0] | f9[1]) | (f9[2] | f9[3]);
+                    if (a2 | a9) {  // exact pass (rare); chunks arrive out of order: ties go to the smaller index
+#pragma unroll 1
+                        for (int u = 0; u < U; ++u) {
+                            const uint32_t cand = chunk * U + u;
+                            const double q = cQ[cand];
+#pragma unroll
+                            for (int r = 0; r < R; ++r) {
+                                const double t2 = fma(pm1[r], q, L), t9 = fma(lf[r], q, lcL[r]);
+                                if (t2 < st2[r] || (t2 == st2[r] && cand < si2[r])) { st2[r] = t2; si2[r] = cand; }
+                                if (t9 < st9[r] || (t9 == st9[r] && cand < si9[r])) { st9[r] = t9; si9[r] = cand; }
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < U; ++u) cur[u] = nxt[u];
+                    chunk = next;
+                }
+                if (ns == 0) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) si2[r] = si9[r] = kSiWhole;
+                }
+                consider(2, st2, si2);
+            };
             // ids 2 and 9 are a_P * Q(s) + c_P with a_P > 0: their best candidate is the same for every P
             const int cpQ = (pilotQ >> (4 * mi)) & 15;
 
@@ -257,7 +320,9 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 for (int r = 0; r < R; ++r) v[r] = fma(pm1[r], gm, rdv);
                 consider(1, v, nullptr);
             }
-            if ((mask >> 2) & 1u)  // Segmented Flat Tree
+            const bool both29 = ((mask >> 2) & 1u) && ((mask >> 9) & 1u);
+            if (both29) segmented_2_and_9(cpQ);
+            else if ((mask >> 2) & 1u)  // Segmented Flat Tree
                 segmented(2, cpQ, [&](int cand) { return cQ[cand]; }, [&](int r, double q) { return fma(pm1[r], q, L); });
             if ((mask >> 3) & 1u) {  // Chain
 #pragma unroll
@@ -288,7 +353,8 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 for (int r = 0; r < R; ++r) v[r] = fma(lf[r], gm, lc[r] * rdv);
                 consider(8, v, nullptr);
             }
-            if ((mask >> 9) & 1u)  // Segmented Binomial Tree
+            if (both29) consider(9, st9, si9);
+            else if ((mask >> 9) & 1u)  // Segmented Binomial Tree
                 segmented(9, cpQ, [&](int cand) { return cQ[cand]; }, [&](int r, double q) { return fma(lf[r], q, lcL[r]); });
 
 #pragma unroll
