@@ -33,7 +33,7 @@ NOMINAL_FP64_FMA_RATE = 148 * 64 * 1.965e9  # SMs x FP64 lanes per SM x max SM c
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (reduced cfg4 with 256 tables; output bytes grow in proportion to the table count, so a full launch of
 # 4096 tables is 16 x the captured one).  Set an entry to None when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_TABLE = {"decide_kernel": (162.75e6 + 0.45e6) / 256, "scatter_kernel": (159.08e6 + 0.94e6) / 256,
+NCU_TRAFFIC_BYTES_PER_TABLE = {"decide_kernel": (163.57e6 + 0.47e6) / 256, "scatter_kernel": (159.08e6 + 0.94e6) / 256,
                                "sweep_kernel": None}
 FALLBACK_HBM_GBS = 6650.0
 
