@@ -211,7 +211,7 @@ def run_reference(args, rank):
         "impl": "reference", "metric": "model_cells_per_sec", "value": value, "unit": "cells/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.model_cells() / value,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "note": "CPU oracle on a bounded sample; ms_per_step extrapolates to the full step"},
+        "config": {"workload": w.name, "call": "plogp_predict" if predict else "plogp_select_best", "note": "CPU oracle on a bounded sample; ms_per_step extrapolates to the full step"},
         "cpu_baseline": {"value": value, "unit": "cells/s", "cores": cores, "kind": "oracle", "sample": text},
         "e2e": {"value": value, "unit": "cells/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
@@ -226,6 +226,8 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--scale", default="full", choices=["full", "small"], help="small: reduced copy for profiler captures")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--call", default="select_best", choices=["select_best", "predict"],
+                    help="predict: time plogp_predict (all model planes) instead of the decision table; device-resident only")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
 
@@ -255,14 +257,34 @@ def main():
     counts = work_counts(w)
     grid = plogp.GridArgs.from_workload(w)
     tabs = plogp.Tables.from_workload(w)
-    out = plogp.alloc_decision(w.n_tables, w.n_P, w.n_m)
-    out_bytes = out.strategy.numel() * 13
+    predict = args.call == "predict"
+    if predict:
+        # all enabled model planes (8 B) plus the best segment size of each segmented strategy (4 B)
+        out = plogp.predict(tabs, grid)
+        torch.cuda.synchronize()
+        n_on = bin(w.strategy_mask).count("1")
+        n_seg = sum((w.strategy_mask >> b) & 1 for b in (2, 5, 9))
+        out_bytes = w.n_tables * w.n_P * w.n_m * (8 * n_on + 4 * n_seg)
+        slots = counts["fp64_slots"]
+        if "sweep_kernel" in counts["per_kernel"]:
+            counts["per_kernel"] = {"sweep_kernel": counts["per_kernel"]["sweep_kernel"],
+                                    "fused_kernel": {"fp64_slots": slots - counts["per_kernel"]["sweep_kernel"]["fp64_slots"], "hbm_bytes": out_bytes}}
+        else:
+            counts["per_kernel"] = {"fused_kernel": {"fp64_slots": slots, "hbm_bytes": out_bytes}}
+        counts["hbm_bytes"] = out_bytes
+        args.e2e_steps = 0
+    else:
+        out = plogp.alloc_decision(w.n_tables, w.n_P, w.n_m)
+        out_bytes = out.strategy.numel() * 13
     flush = None
     if out_bytes < (256 << 20):  # outputs do not evict the 126 MB L2 by themselves: write 256 MB between steps
         flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
     def step():
-        plogp.select_best(tabs, grid, out=out)
+        if predict:
+            plogp.predict(tabs, grid, out=out)
+        else:
+            plogp.select_best(tabs, grid, out=out)
 
     for _ in range(args.warmup):
         step()
@@ -363,7 +385,7 @@ def main():
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "decision_cells_per_sec": world * counts["decision_cells"] / step_s,
-        "config": {"workload": w.name, "tables_per_gpu": w.n_tables, "P": [w.P_lo, w.P_hi], "n_m": w.n_m,
+        "config": {"workload": w.name, "call": "plogp_predict" if predict else "plogp_select_best", "tables_per_gpu": w.n_tables, "P": [w.P_lo, w.P_hi], "n_m": w.n_m,
                    "n_s": int(len(w.s_values())), "strategy_mask": w.strategy_mask, "model_cells_per_gpu": counts["model_cells"],
                    "decision_cells_per_gpu": counts["decision_cells"], "parallelism": "tables sharded, %d rank(s)" % world,
                    "l2": ("outputs (%.1f GB per step) exceed the 126 MB L2" % (out_bytes / 1e9)) if flush is None
