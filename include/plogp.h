@@ -61,7 +61,7 @@ typedef enum {
     PLOGP_E_NOMEM = -2, /* host or device allocation failed */
     PLOGP_E_CUDA = -3,  /* a CUDA runtime call failed; plogp_last_cuda_error() names it */
     PLOGP_E_RANGE = -4  /* m, s or a table size too large: m and s must be < 2^32, sizes < 2^53,
-                           n_bp <= PLOGP_MAX_BREAKPOINTS, (P_hi - 1) * m < 2^53 */
+                           n_bp <= PLOGP_MAX_BREAKPOINTS, P_hi * m < 2^53 (so that j * m is exact in a double) */
 } plogp_status;
 
 /* Opaque set of pLogP parameter tables resident on the current CUDA device. */
