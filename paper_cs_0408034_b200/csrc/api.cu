@@ -260,9 +260,10 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     pl.n_ptiles = (total_passes + pl.passes_per_tile - 1) / pl.passes_per_tile;
 
     pl.dec_ptiles = (n_P + kDecTileP - 1) / kDecTileP;
-    // 8 message sizes per CTA give the widest output rows; small grids trade that for more CTAs
+    // 16 message sizes per CTA give the widest output rows; small grids trade that for more CTAs
+    // (never fewer than one message size per warp)
     pl.dec_mg = kDecMG;
-    while (pl.dec_mg > 1 && (long long)((n_m + pl.dec_mg - 1) / pl.dec_mg) * pl.dec_ptiles * h->T.n_tables < (long long)h->sm_count * 4)
+    while (pl.dec_mg > kDecWarps && (long long)((n_m + pl.dec_mg - 1) / pl.dec_mg) * pl.dec_ptiles * h->T.n_tables < (long long)h->sm_count * 4)
         pl.dec_mg >>= 1;
     pl.dec_mgroups = (n_m + pl.dec_mg - 1) / pl.dec_mg;
 

@@ -2,18 +2,28 @@
 // candidate lists, with lanes mapped to the process count P.  (The Scatter half has no candidate
 // lists and goes through scatter_kernel.)
 //
-// One CTA owns one table, a group of 8 message sizes and a tile of 512 process counts (4 warps x
-// 32 lanes x 4 cells).  For a fixed (m, s) the segmented models of Table 1 are lines in P, so the
-// CTA computes the line coefficients once per (m, s) into shared memory and every lane reads them
-// with one broadcast load.  Each model cell is evaluated with one DFMA.  The comparison with the
-// running minimum is first made on the high 32 bits in the integer pipe (times are non-negative,
-// so a smaller double never has a larger high word); only chunks of candidates in which some cell
-// can improve run the exact FP64 compare-and-select pass.  To make that pass rare, each warp first
-// finds the best candidate for the process count in the middle of its range (one candidate per
-// lane, one warp-wide integer minimum over float keys) and evaluates that candidate's chunk first: neighbouring process counts
-// nearly always share the optimum, and for ids 2 and 9 the optimum does not depend on P at all.
+// One CTA owns one table, a group of up to 16 message sizes and a tile of 256 process counts.  All
+// four warps work on the same 256 process counts (lane + 32 r, r = 0..7) and split the message
+// sizes, so a warp runs on its own from the candidate lists to the staged result and only the
+// write-out needs the whole CTA.
 //
-// Results are staged in shared memory as [m][P] and written out as rows of 8 consecutive m.
+// Every model of Table 1 is, for a fixed message size (and segment size), a line in P or in
+// floor(log2 P):
+//     ids 0 1 2 3 4 5:  t = fma(P-1, a, c)           "P list", entries (a, c)
+//     ids 7 9:          t = fma(floor(log2 P), a, ceil(log2 P) L)   "log list", entries a
+//     ids 6 8:          one cell each, evaluated on their own
+// The decision is the lexicographic minimum of (t, id, s) over all cells of all enabled strategies
+// (the minimum over s inside a strategy and then over strategies, smallest s and lowest id on
+// ties), so one running minimum per process count serves the whole search.  A warp builds the two
+// lists of a message size in shared memory (lanes <-> candidates), guesses the winner at the
+// process count in the middle of its range (the pilot), starts the running minimum from the
+// pilot's cells and takes the pilot out of its list.  Then every cell is evaluated with one DFMA
+// and compared with the running minimum on the high 32 bits only, in the integer pipe (times are
+// non-negative, so a smaller double never has a larger high word); a group of four list entries in
+// which some cell can reach the minimum is re-evaluated with the exact FP64 comparison, for the
+// eight-cell rows that need it.  With a good pilot that is rare.
+//
+// Results are staged in shared memory as [m][P] and written out as rows of consecutive m.
 #include "device_common.cuh"
 
 #include <algorithm>
@@ -22,44 +32,60 @@ namespace plogp {
 
 namespace {
 
-constexpr int kDecStride = kDecTileP + 2;  // doubles per staged row: keeps the transposed reads conflict-free
+constexpr int R = kDecR, U = kDecU;
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kStageStride = kDecTileP + 1;  // doubles per staged row: the transposed reads stay conflict-free
+constexpr int kCodeStride = kDecTileP + 2;   // 16-bit codes per staged row, for the same reason
+
+constexpr uint32_t kCandNone = 255;   // winner is an unsegmented strategy
+constexpr uint32_t kCandWhole = 254;  // segmented winner with no fitting candidate: the whole message
+constexpr uint32_t kCodeNever = 0xFFFFu;
+constexpr unsigned kNoPilot = 0x1FFu;
 
 struct DecSmem {
-    double *tab, *gs, *cQ, *gm, *st_time;
-    double2 *cBC;
-    uint8_t *st_id, *st_si;
+    double *tab, *gs, *gm, *lf, *lc, *l2, *st_time;
+    double2 *l1;
+    uint32_t *sval;
+    uint16_t *c1, *c2, *st_code;
+    int cap1, cap2;
 };
 
-__host__ __device__ inline size_t dec_layout(int npad, int nsp, unsigned char *base, DecSmem *o)
+__host__ __device__ inline int round_up(int x, int a) { return (x + a - 1) / a * a; }
+
+// Shared-memory layout.  cap1 / cap2: entries of one warp's P list / log list (multiples of U).
+__host__ __device__ inline size_t dec_layout(int npad, int n_s, unsigned char *base, DecSmem *o)
 {
+    const int nsv = n_s > 0 ? n_s : 1;
+    const int cap1 = round_up(2 * nsv + 4, U), cap2 = round_up(nsv + 1, U);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off += (bytes + 15) & ~size_t(15); return at; };
-    const size_t o_tab = take(3 * size_t(npad) * 8), o_gs = take(size_t(nsp) * 8), o_BC = take(size_t(kDecMG) * nsp * 16),
-                 o_Q = take(size_t(kDecMG) * nsp * 8), o_gm = take(kDecMG * 8), o_t = take(size_t(kDecMG) * kDecStride * 8),
-                 o_id = take(size_t(kDecMG) * (kDecTileP + 16)), o_si = take(size_t(kDecMG) * (kDecTileP + 16));
+    const size_t o_tab = take(3 * size_t(npad) * 8), o_gs = take(size_t(nsv) * 8), o_sv = take(size_t(nsv) * 4),
+                 o_gm = take(kDecMG * 8), o_lf = take(kDecTileP * 8), o_lc = take(kDecTileP * 8),
+                 o_l1 = take(size_t(kDecWarps) * cap1 * 16), o_l2 = take(size_t(kDecWarps) * cap2 * 8),
+                 o_c1 = take(size_t(kDecWarps) * cap1 * 2), o_c2 = take(size_t(kDecWarps) * cap2 * 2),
+                 o_t = take(size_t(kDecMG) * kStageStride * 8), o_c = take(size_t(kDecMG) * kCodeStride * 2);
     if (o) {
         o->tab = reinterpret_cast<double *>(base + o_tab); o->gs = reinterpret_cast<double *>(base + o_gs);
-        o->cBC = reinterpret_cast<double2 *>(base + o_BC); o->cQ = reinterpret_cast<double *>(base + o_Q);
-        o->gm = reinterpret_cast<double *>(base + o_gm); o->st_time = reinterpret_cast<double *>(base + o_t);
-        o->st_id = base + o_id; o->st_si = base + o_si;
+        o->sval = reinterpret_cast<uint32_t *>(base + o_sv); o->gm = reinterpret_cast<double *>(base + o_gm);
+        o->lf = reinterpret_cast<double *>(base + o_lf); o->lc = reinterpret_cast<double *>(base + o_lc);
+        o->l1 = reinterpret_cast<double2 *>(base + o_l1); o->l2 = reinterpret_cast<double *>(base + o_l2);
+        o->c1 = reinterpret_cast<uint16_t *>(base + o_c1); o->c2 = reinterpret_cast<uint16_t *>(base + o_c2);
+        o->st_time = reinterpret_cast<double *>(base + o_t); o->st_code = reinterpret_cast<uint16_t *>(base + o_c);
+        o->cap1 = cap1; o->cap2 = cap2;
     }
     return off;
 }
 
-constexpr uint8_t kSiNone = 255;      // winner is an unsegmented strategy
-constexpr uint8_t kSiWhole = 254;     // segmented winner with no fitting candidate: the whole message
-
+__device__ __forceinline__ int hi32(double x) { return __double2hiint(x); }
 
 }  // namespace
 
 __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecideParams p)
 {
-    constexpr int R = kDecR, U = kDecU;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int npad = p.T.npad;
-    const int nsp = (max(p.G.n_s, 1) + U - 1) / U * U;
     DecSmem sm;
-    dec_layout(npad, nsp, smem_raw, &sm);
+    dec_layout(npad, p.G.n_s, smem_raw, &sm);
     const uint32_t mask = p.G.mask;
 
     int b = blockIdx.x;
@@ -69,14 +95,25 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     const int trel = b / p.n_ptiles;
     const int table = p.table0 + trel;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int m0 = mgroup * p.mg;   // p.mg <= kDecMG message sizes per CTA (fewer on small grids, for more CTAs)
+    const int m0 = mgroup * p.mg;  // p.mg <= kDecMG message sizes per CTA (fewer on small grids, for more CTAs)
     const int n_mi = min(p.mg, p.G.n_m - m0);
+    const int tile0 = ptile * kDecTileP;
+    const int n_valid = min(kDecTileP, p.G.n_P - tile0);
 
     stage_table(sm.tab, p.T, table);
+    // floor(log2 P) and ceil(log2 P) of the tile's process counts, as doubles
+    for (int i = tid; i < kDecTileP; i += kDecThreads) {
+        const int P = P_at(p.G, min(tile0 + i, p.G.n_P - 1));
+        sm.lf[i] = static_cast<double>(31 - __clz(P));
+        sm.lc[i] = static_cast<double>(32 - __clz(P - 1));
+    }
     __syncthreads();
     const double L = p.T.lat[table];
-    for (int si = tid; si < p.G.n_s; si += kDecThreads)
-        sm.gs[si] = gap_at(sm.tab, npad, static_cast<double>(s_at(p.G, si)));
+    for (int si = tid; si < p.G.n_s; si += kDecThreads) {
+        const uint32_t s = s_at(p.G, si);
+        sm.sval[si] = s;
+        sm.gs[si] = gap_at(sm.tab, npad, static_cast<double>(s));
+    }
     if (tid >= kDecThreads - kDecMG) {  // g(m) of the group's message sizes, by the last threads
         const int mi = tid - (kDecThreads - kDecMG);
         if (mi < n_mi) sm.gm[mi] = gap_at(sm.tab, npad, static_cast<double>(p.G.m_list[m0 + mi]));
@@ -84,297 +121,240 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     const double g1 = gap_at(sm.tab, npad, 1.0);
     const double rdv = 2.0 * g1 + 3.0 * L;  // rendezvous handshake: 2 g(1) + 3 L
     __syncthreads();
-    // line coefficients per (message size of the group, candidate): Section 2's k, Table 1's segmented rows
-    for (int idx = tid; idx < n_mi * nsp; idx += kDecThreads) {
-        const int mi = idx / nsp, si = idx - mi * nsp;
-        const uint32_t m_u = p.G.m_list[m0 + mi];
-        const int ns = p.G.ns_of_m[m0 + mi];
-        double B = CUDART_INF, C = CUDART_INF, Q = CUDART_INF;  // padding never wins
-        if (si < ns) {
-            const double gs = sm.gs[si];
-            const double k = static_cast<double>(segments(m_u, s_at(p.G, si), p.G.k_mode));
-            B = gs + L; C = gs * (k - 1.0); Q = gs * k;
-        } else if (ns == 0 && si == 0) {  // nothing fits: the whole message, k = 1
-            B = sm.gm[mi] + L; C = 0.0; Q = sm.gm[mi];
+
+    // this thread's cells: process counts at tile offset 32 r + lane
+    double pm1[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) pm1[r] = static_cast<double>(P_at(p.G, min(tile0 + 32 * r + lane, p.G.n_P - 1)) - 1);
+    // the pilot's process count: middle of the tile's valid range
+    const int P_mid = P_at(p.G, tile0 + n_valid / 2);
+    const double x1_mid = static_cast<double>(P_mid - 1);
+    const double x2_mid = static_cast<double>(31 - __clz(P_mid));
+    const double c2_mid = static_cast<double>(32 - __clz(P_mid - 1)) * L;
+
+    const uint32_t un = mask & 0x1Bu;  // unsegmented members of the P list: ids 0, 1, 3, 4
+    const int n_un = __popc(un);
+    const bool has2 = (mask >> 2) & 1u, has5 = (mask >> 5) & 1u, has6 = (mask >> 6) & 1u, has7 = (mask >> 7) & 1u,
+               has8 = (mask >> 8) & 1u, has9 = (mask >> 9) & 1u;
+    double2 *l1 = sm.l1 + warp * sm.cap1;
+    double *l2 = sm.l2 + warp * sm.cap2;
+    uint16_t *c1 = sm.c1 + warp * sm.cap1, *c2 = sm.c2 + warp * sm.cap2;
+
+    for (int mi = warp; mi < n_mi; mi += kDecWarps) {
+        const int midx = m0 + mi;
+        const uint32_t m_u = p.G.m_list[midx];
+        const int ns = p.G.ns_of_m[midx];
+        const int nsv = max(ns, 1);  // candidates actually evaluated (none fits: the whole message, k = 1)
+        const double gm = sm.gm[mi];
+        const int o2 = n_un, o5 = o2 + (has2 ? nsv : 0), n1 = o5 + (has5 ? nsv : 0);
+        const int o9 = has7 ? 1 : 0, n2 = o9 + (has9 ? nsv : 0);
+        const int n1p = round_up(n1, U), n2p = round_up(n2, U);
+
+        // ---- the two lists of this message size, and each lane's best entry at the pilot's process count ----
+        __syncwarp();  // the previous message size's loops have finished reading the lists
+        double tb = CUDART_INF;
+        unsigned pb = kNoPilot;  // P-list position, or 256 + log-list position
+        auto offer = [&](double t, unsigned pos) {
+            if (t < tb) { tb = t; pb = pos; }
+        };
+        if (lane < 4) {
+            const int id = lane + (lane >> 1);  // 0, 1, 3, 4
+            if ((mask >> id) & 1u) {
+                const int pos = __popc(un & ((1u << id) - 1u));
+                // Flat Tree (P-1) g + L, its rendezvous form (P-1) g + rdv; Chain (P-1)(g + L), rendezvous (P-1)(g + rdv)
+                const double a = id >= 3 ? gm + (id == 4 ? rdv : L) : gm;
+                const double c = id >= 3 ? 0.0 : (id == 1 ? rdv : L);
+                l1[pos] = make_double2(a, c);
+                c1[pos] = static_cast<uint16_t>((id << 8) | kCandNone);
+                offer(fma(x1_mid, a, c), pos);
+            }
         }
-        sm.cBC[idx] = make_double2(B, C);
-        sm.cQ[idx] = Q;
+        if (lane == 4 && has7) {  // Binomial Tree
+            l2[0] = gm;
+            c2[0] = static_cast<uint16_t>((7u << 8) | kCandNone);
+            offer(fma(x2_mid, gm, c2_mid), 256u);
+        }
+        for (int i = n1 + lane; i < n1p; i += 32) {  // padding never reaches the minimum
+            l1[i] = make_double2(CUDART_INF, CUDART_INF);
+            c1[i] = static_cast<uint16_t>(kCodeNever);
+        }
+        for (int i = n2 + lane; i < n2p; i += 32) {
+            l2[i] = CUDART_INF;
+            c2[i] = static_cast<uint16_t>(kCodeNever);
+        }
+        for (int c = lane; c < nsv; c += 32) {
+            // Section 2's k and the line coefficients of Table 1's segmented rows
+            double gsv = gm, k = 1.0;
+            uint32_t cand = kCandWhole;
+            if (ns > 0) {
+                gsv = sm.gs[c];
+                k = static_cast<double>(segments(m_u, sm.sval[c], p.G.k_mode));
+                cand = static_cast<uint32_t>(c);
+            }
+            const double Q = gsv * k;
+            if (has2) {  // (P-1) (g(s) k) + L
+                l1[o2 + c] = make_double2(Q, L);
+                c1[o2 + c] = static_cast<uint16_t>((2u << 8) | cand);
+                offer(fma(x1_mid, Q, L), o2 + c);
+            }
+            if (has5) {  // (P-1) (g(s) + L) + g(s) (k-1)
+                const double B = gsv + L, C = gsv * (k - 1.0);
+                l1[o5 + c] = make_double2(B, C);
+                c1[o5 + c] = static_cast<uint16_t>((5u << 8) | cand);
+                offer(fma(x1_mid, B, C), o5 + c);
+            }
+            if (has9) {  // floor(log2 P) g(s) k + ceil(log2 P) L
+                l2[o9 + c] = Q;
+                c2[o9 + c] = static_cast<uint16_t>((9u << 8) | cand);
+                offer(fma(x2_mid, Q, c2_mid), 256u + o9 + c);
+            }
+        }
+        // warp-wide pilot: smallest time (high word first, then low word with the position in its last 9 bits)
+        const int hmin = __reduce_min_sync(kFull, hi32(tb));
+        const unsigned k2 = hi32(tb) == hmin ? ((static_cast<unsigned>(__double2loint(tb)) & ~0x1FFu) | pb) : 0xFFFFFFFFu;
+        const unsigned pilot = __reduce_min_sync(kFull, k2) & 0x1FFu;
+        __syncwarp();
+
+        double lf[R], lcL[R];  // floor(log2 P); ceil(log2 P), later ceil(log2 P) L
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            lf[r] = sm.lf[32 * r + lane];
+            lcL[r] = sm.lc[32 * r + lane];
+        }
+
+        // ---- running minimum per process count, started from the pilot's cells ----
+        double bt[R];
+        uint32_t bcode[R];  // strategy id << 8 | candidate index (or kCandNone / kCandWhole)
+        if (pilot == kNoPilot) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) { bt[r] = CUDART_INF; bcode[r] = kCodeNever; }
+        } else if (pilot < 256u) {
+            const double2 e = l1[pilot];
+            const uint32_t code = c1[pilot];
+            __syncwarp();
+            if (lane == 0) l1[pilot] = make_double2(CUDART_INF, CUDART_INF);
+#pragma unroll
+            for (int r = 0; r < R; ++r) { bt[r] = fma(pm1[r], e.x, e.y); bcode[r] = code; }
+        } else {
+            const double a = l2[pilot - 256u];
+            const uint32_t code = c2[pilot - 256u];
+            __syncwarp();
+            if (lane == 0) l2[pilot - 256u] = CUDART_INF;
+#pragma unroll
+            for (int r = 0; r < R; ++r) { bt[r] = fma(lf[r], a, lcL[r] * L); bcode[r] = code; }
+        }
+        __syncwarp();
+
+        // one cell per process count (ids 6 and 8): high-word test, exact comparison where it holds
+        auto single = [&](uint32_t code, const double *t) {
+            bool f[R], any = false;
+#pragma unroll
+            for (int r = 0; r < R; ++r) { f[r] = hi32(t[r]) <= hi32(bt[r]); any |= f[r]; }
+            if (any) {
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+                    if (f[r] && (t[r] < bt[r] || (t[r] == bt[r] && code < bcode[r]))) { bt[r] = t[r]; bcode[r] = code; }
+            }
+        };
+        if (has6) {  // Binary Tree (the printed bound): ceil(log2 P) (2 g(m) + L)
+            const double w = fma(2.0, gm, L);
+            double t[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) t[r] = lcL[r] * w;
+            single((6u << 8) | kCandNone, t);
+        }
+        if (has8) {  // Binomial Tree Rendezvous: floor(log2 P) g(m) + ceil(log2 P) rdv
+            double t[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) t[r] = fma(lf[r], gm, lcL[r] * rdv);
+            single((8u << 8) | kCandNone, t);
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) lcL[r] *= L;
+
+        // ---- log list: t = fma(floor(log2 P), a, ceil(log2 P) L) ----
+#pragma unroll 1
+        for (int j = 0; j < n2p; j += U) {
+            const double2 q01 = *reinterpret_cast<const double2 *>(l2 + j), q23 = *reinterpret_cast<const double2 *>(l2 + j + 2);
+            bool f[R], any = false;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int h0 = hi32(fma(lf[r], q01.x, lcL[r])), h1 = hi32(fma(lf[r], q01.y, lcL[r]));
+                const int h2 = hi32(fma(lf[r], q23.x, lcL[r])), h3 = hi32(fma(lf[r], q23.y, lcL[r]));
+                f[r] = min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]);
+                any |= f[r];
+            }
+            if (__any_sync(kFull, any)) {  // rare: exact comparison, (time, id, candidate) in lexicographic order
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    if (__any_sync(kFull, f[r])) {
+#pragma unroll 1
+                        for (int u = 0; u < U; ++u) {
+                            const double t = fma(lf[r], l2[j + u], lcL[r]);
+                            const uint32_t code = c2[j + u];
+                            if (t < bt[r] || (t == bt[r] && code < bcode[r])) { bt[r] = t; bcode[r] = code; }
+                        }
+                    }
+                }
+            }
+        }
+
+        // ---- P list: t = fma(P-1, a, c) ----
+#pragma unroll 1
+        for (int j = 0; j < n1p; j += U) {
+            const double2 e0 = l1[j], e1 = l1[j + 1], e2 = l1[j + 2], e3 = l1[j + 3];
+            bool f[R], any = false;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int h0 = hi32(fma(pm1[r], e0.x, e0.y)), h1 = hi32(fma(pm1[r], e1.x, e1.y));
+                const int h2 = hi32(fma(pm1[r], e2.x, e2.y)), h3 = hi32(fma(pm1[r], e3.x, e3.y));
+                f[r] = min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]);
+                any |= f[r];
+            }
+            if (__any_sync(kFull, any)) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    if (__any_sync(kFull, f[r])) {
+#pragma unroll 1
+                        for (int u = 0; u < U; ++u) {
+                            const double2 e = l1[j + u];
+                            const double t = fma(pm1[r], e.x, e.y);
+                            const uint32_t code = c1[j + u];
+                            if (t < bt[r] || (t == bt[r] && code < bcode[r])) { bt[r] = t; bcode[r] = code; }
+                        }
+                    }
+                }
+            }
+        }
+
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            sm.st_time[mi * kStageStride + 32 * r + lane] = bt[r];
+            sm.st_code[mi * kCodeStride + 32 * r + lane] = static_cast<uint16_t>(bcode[r]);
+        }
     }
     __syncthreads();
 
-    // this thread's cells: process counts at tile offset warp*128 + r*32 + lane
-    const int p_first = ptile * kDecTileP + warp * (32 * R) + lane;
-    int Pv[R];
-    double pm1[R], lf[R], lc[R], lcL[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const int pidx = p_first + 32 * r;
-        Pv[r] = P_at(p.G, min(pidx, p.G.n_P - 1));
-        pm1[r] = static_cast<double>(Pv[r] - 1);
-        lf[r] = static_cast<double>(31 - __clz(Pv[r]));
-        lc[r] = static_cast<double>(32 - __clz(Pv[r] - 1));
-        lcL[r] = lc[r] * L;
-    }
-    // the warp's pilot process count (middle of its range, clamped to the grid)
-    const int P_mid = P_at(p.G, min(ptile * kDecTileP + warp * (32 * R) + 16 * R, p.G.n_P - 1));
-    const double pm1_mid = static_cast<double>(P_mid - 1);
-
-    // Pilots for the whole group, issued together so that their latencies overlap: for each message size
-    // the chunk holding the candidate that is best at the warp's middle process count.  Only a guess that
-    // orders the work (float precision, candidate index in the low bits of the key); 4 bits per message size.
-    uint32_t pilotQ = 0, pilot5 = 0;
-    if (mask & ((1u << 2) | (1u << 5) | (1u << 9))) {
-#pragma unroll
-        for (int mi = 0; mi < kDecMG; ++mi) {
-            if (mi < n_mi) {
-                const int nsv = max(p.G.ns_of_m[m0 + mi], 1);
-                unsigned kq = 0xFFFFFFFFu, k5 = 0xFFFFFFFFu;
-                for (int c0 = 0; c0 < nsv; c0 += 32) {
-                    const int cand = c0 + lane;
-                    if (cand < nsv) {
-                        const double2 c = sm.cBC[mi * nsp + cand];
-                        kq = min(kq, (__float_as_uint(static_cast<float>(sm.cQ[mi * nsp + cand])) & ~63u) | static_cast<unsigned>(cand));
-                        k5 = min(k5, (__float_as_uint(static_cast<float>(fma(pm1_mid, c.x, c.y))) & ~63u) | static_cast<unsigned>(cand));
-                    }
-                }
-                pilotQ |= ((__reduce_min_sync(0xffffffffu, kq) & 63u) / U) << (4 * mi);
-                pilot5 |= ((__reduce_min_sync(0xffffffffu, k5) & 63u) / U) << (4 * mi);
-            }
-        }
-    }
-
-    const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
-
-    // transposed write-out of the staged group: rows of n_mi consecutive m per process count
-    auto write_out = [&](int coll) {
-        const int mi = lane & 7, prow = lane >> 3;
+    // transposed write-out of the staged group: rows of p.mg consecutive m per process count
+    {
+        const int mi = lane & (p.mg - 1), prow = lane / p.mg, rows = 32 / p.mg;
         if (mi < n_mi) {
             const uint32_t m_u = p.G.m_list[m0 + mi];
-            for (int pr = warp * 4 + prow; pr < kDecTileP; pr += kDecWarps * 4) {
-                const int pidx = ptile * kDecTileP + pr;
-                if (pidx >= p.G.n_P) break;
-                const size_t o = (static_cast<size_t>(table) * 2 + coll) * plane + static_cast<size_t>(pidx) * p.G.n_m + m0 + mi;
-                const uint8_t si = sm.st_si[mi * (kDecTileP + 16) + pr];
-                p.d_time[o] = sm.st_time[mi * kDecStride + pr];
-                p.d_strategy[o] = sm.st_id[mi * (kDecTileP + 16) + pr];
-                p.d_sbytes[o] = si == kSiNone ? 0u : (si == kSiWhole ? m_u : s_at(p.G, si));
+            const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
+            const size_t base = static_cast<size_t>(table) * 2 * plane + static_cast<size_t>(m0 + mi);
+            for (int pr = warp * rows + prow; pr < n_valid; pr += kDecWarps * rows) {
+                const size_t o = base + static_cast<size_t>(tile0 + pr) * p.G.n_m;
+                const uint32_t code = sm.st_code[mi * kCodeStride + pr];
+                const uint32_t cand = code & 255u;
+                p.d_time[o] = sm.st_time[mi * kStageStride + pr];
+                p.d_strategy[o] = static_cast<uint8_t>(code >> 8);
+                p.d_sbytes[o] = cand == kCandNone ? 0u : (cand == kCandWhole ? m_u : sm.sval[cand]);
             }
         }
-    };
-
-    // =============================== Broadcast (Table 1) ===============================
-    if (mask & 0x3FFu) {
-        for (int mi = 0; mi < n_mi; ++mi) {
-            const int midx = m0 + mi;
-            const int ns = p.G.ns_of_m[midx];
-            const int nsv = max(ns, 1);                 // candidates actually evaluated
-            const int n_chunks = (nsv + U - 1) / U;
-
-            const double gm = sm.gm[mi];
-            const double2 *cBC = sm.cBC + mi * nsp;
-            const double *cQ = sm.cQ + mi * nsp;
-
-            double bt[R];
-            uint32_t bcode[R];  // winner so far: strategy id << 8 | candidate index (or kSiNone / kSiWhole)
-#pragma unroll
-            for (int r = 0; r < R; ++r) { bt[r] = CUDART_INF; bcode[r] = (255u << 8) | kSiNone; }
-            auto consider = [&](int id, const double *val, const uint32_t *sval) {
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-                    if (val[r] < bt[r]) { bt[r] = val[r]; bcode[r] = (static_cast<uint32_t>(id) << 8) | (sval ? sval[r] : kSiNone); }
-            };
-
-            // Segmented model reduced over the candidates: load(cand) fetches the candidate's line
-            // coefficients from shared memory, eval(r, coef) is the model cell.
-            auto segmented = [&](int id, int cp, auto load, auto eval) {
-                double st[R];
-                uint32_t si[R];
-#pragma unroll
-                for (int r = 0; r < R; ++r) { st[r] = CUDART_INF; si[r] = 0; }
-                // the pilot's chunk first, ascending, strict '<'
-#pragma unroll 1
-                for (int u = 0; u < U; ++u) {
-                    const uint32_t cand = cp * U + u;
-                    const auto k = load(cand);
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        const double t = eval(r, k);
-                        if (t < st[r]) { st[r] = t; si[r] = cand; }
-                    }
-                }
-                // all other chunks; the next chunk's coefficients are fetched before the current one is tested
-                decltype(load(0)) cur[U], nxt[U];
-                int chunk = cp == 0 ? 1 : 0;
-#pragma unroll
-                for (int u = 0; u < U; ++u) cur[u] = load(min(chunk, n_chunks - 1) * U + u);
-                while (chunk < n_chunks) {
-                    int next = chunk + 1;
-                    next += next == cp;
-#pragma unroll
-                    for (int u = 0; u < U; ++u) nxt[u] = load(min(next, n_chunks - 1) * U + u);
-                    // one flag per cell: a single flag would chain all 16 integer compares through one predicate
-                    bool f[R];
-#pragma unroll
-                    for (int r = 0; r < R; ++r) f[r] = false;
-#pragma unroll
-                    for (int u = 0; u < U; ++u) {
-#pragma unroll
-                        for (int r = 0; r < R; ++r)
-                            f[r] |= __double2hiint(eval(r, cur[u])) <= __double2hiint(st[r]);
-                    }
-                    if ((f[0] | f[1]) | (f[2] | f[3])) {  // exact pass; chunks arrive out of order: ties go to the smaller index
-#pragma unroll
-                        for (int u = 0; u < U; ++u) {
-                            const uint32_t cand = chunk * U + u;
-#pragma unroll
-                            for (int r = 0; r < R; ++r) {
-                                const double t = eval(r, cur[u]);
-                                if (t < st[r] || (t == st[r] && cand < si[r])) { st[r] = t; si[r] = cand; }
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < U; ++u) cur[u] = nxt[u];
-                    chunk = next;
-                }
-                if (ns == 0) {
-#pragma unroll
-                    for (int r = 0; r < R; ++r) si[r] = kSiWhole;
-                }
-                consider(id, st, si);
-            };
-            // Ids 2 and 9 together: both read Q(s), so one sweep loads it once and tests 32 cells per branch.
-            double st9[R];
-            uint32_t si9[R];
-            auto segmented_2_and_9 = [&](int cp) {
-                double st2[R];
-                uint32_t si2[R];
-#pragma unroll
-                for (int r = 0; r < R; ++r) { st2[r] = st9[r] = CUDART_INF; si2[r] = si9[r] = 0; }
-#pragma unroll 1
-                for (int u = 0; u < U; ++u) {  // the pilot's chunk first, ascending, strict '<'
-                    const uint32_t cand = cp * U + u;
-                    const double q = cQ[cand];
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        const double t2 = fma(pm1[r], q, L), t9 = fma(lf[r], q, lcL[r]);
-                        if (t2 < st2[r]) { st2[r] = t2; si2[r] = cand; }
-                        if (t9 < st9[r]) { st9[r] = t9; si9[r] = cand; }
-                    }
-                }
-                double cur[U], nxt[U];
-                int chunk = cp == 0 ? 1 : 0;
-#pragma unroll
-                for (int u = 0; u < U; ++u) cur[u] = cQ[min(chunk, n_chunks - 1) * U + u];
-                while (chunk < n_chunks) {
-                    int next = chunk + 1;
-                    next += next == cp;
-#pragma unroll
-                    for (int u = 0; u < U; ++u) nxt[u] = cQ[min(next, n_chunks - 1) * U + u];
-                    bool f2[R], f9[R];
-#pragma unroll
-                    for (int r = 0; r < R; ++r) f2[r] = f9[r] = false;
-#pragma unroll
-                    for (int u = 0; u < U; ++u) {
-#pragma unroll
-                        for (int r = 0; r < R; ++r) {
-                            f2[r] |= __double2hiint(fma(pm1[r], cur[u], L)) <= __double2hiint(st2[r]);
-                            f9[r] |= __double2hiint(fma(lf[r], cur[u], lcL[r])) <= __double2hiint(st9[r]);
-                        }
-                    }
-                    const bool a2 = (f2[0] | f2[1]) | (f2[2] | f2[3]), a9 = (f9[0] | f9[1]) | (f9[2] | f9[3]);
-                    if (a2 | a9) {  // exact pass (rare); chunks arrive out of order: ties go to the smaller index
-#pragma unroll 1
-                        for (int u = 0; u < U; ++u) {
-                            const uint32_t cand = chunk * U + u;
-                            const double q = cQ[cand];
-#pragma unroll
-                            for (int r = 0; r < R; ++r) {
-                                const double t2 = fma(pm1[r], q, L), t9 = fma(lf[r], q, lcL[r]);
-                                if (t2 < st2[r] || (t2 == st2[r] && cand < si2[r])) { st2[r] = t2; si2[r] = cand; }
-                                if (t9 < st9[r] || (t9 == st9[r] && cand < si9[r])) { st9[r] = t9; si9[r] = cand; }
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < U; ++u) cur[u] = nxt[u];
-                    chunk = next;
-                }
-                if (ns == 0) {
-#pragma unroll
-                    for (int r = 0; r < R; ++r) si2[r] = si9[r] = kSiWhole;
-                }
-                consider(2, st2, si2);
-            };
-            // ids 2 and 9 are a_P * Q(s) + c_P with a_P > 0: their best candidate is the same for every P
-            const int cpQ = (pilotQ >> (4 * mi)) & 15;
-
-            double v[R];
-            if (mask & 1u) {  // Flat Tree
-#pragma unroll
-                for (int r = 0; r < R; ++r) v[r] = fma(pm1[r], gm, L);
-                consider(0, v, nullptr);
-            }
-            if ((mask >> 1) & 1u) {  // Flat Tree Rendezvous
-#pragma unroll
-                for (int r = 0; r < R; ++r) v[r] = fma(pm1[r], gm, rdv);
-                consider(1, v, nullptr);
-            }
-            const bool both29 = ((mask >> 2) & 1u) && ((mask >> 9) & 1u);
-            if (both29) segmented_2_and_9(cpQ);
-            else if ((mask >> 2) & 1u)  // Segmented Flat Tree
-                segmented(2, cpQ, [&](int cand) { return cQ[cand]; }, [&](int r, double q) { return fma(pm1[r], q, L); });
-            if ((mask >> 3) & 1u) {  // Chain
-#pragma unroll
-                for (int r = 0; r < R; ++r) v[r] = pm1[r] * (gm + L);
-                consider(3, v, nullptr);
-            }
-            if ((mask >> 4) & 1u) {  // Chain Rendezvous
-#pragma unroll
-                for (int r = 0; r < R; ++r) v[r] = pm1[r] * (gm + rdv);
-                consider(4, v, nullptr);
-            }
-            if ((mask >> 5) & 1u) {  // Segmented Chain
-                const int cp5 = (pilot5 >> (4 * mi)) & 15;
-                segmented(5, cp5, [&](int cand) { return cBC[cand]; }, [&](int r, double2 c) { return fma(pm1[r], c.x, c.y); });
-            }
-            if ((mask >> 6) & 1u) {  // Binary Tree (the printed bound)
-#pragma unroll
-                for (int r = 0; r < R; ++r) v[r] = lc[r] * fma(2.0, gm, L);
-                consider(6, v, nullptr);
-            }
-            if ((mask >> 7) & 1u) {  // Binomial Tree
-#pragma unroll
-                for (int r = 0; r < R; ++r) v[r] = fma(lf[r], gm, lcL[r]);
-                consider(7, v, nullptr);
-            }
-            if ((mask >> 8) & 1u) {  // Binomial Tree Rendezvous
-#pragma unroll
-                for (int r = 0; r < R; ++r) v[r] = fma(lf[r], gm, lc[r] * rdv);
-                consider(8, v, nullptr);
-            }
-            if (both29) consider(9, st9, si9);
-            else if ((mask >> 9) & 1u)  // Segmented Binomial Tree
-                segmented(9, cpQ, [&](int cand) { return cQ[cand]; }, [&](int r, double q) { return fma(lf[r], q, lcL[r]); });
-
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const int pr = warp * (32 * R) + 32 * r + lane;
-                sm.st_time[mi * kDecStride + pr] = bt[r];
-                sm.st_id[mi * (kDecTileP + 16) + pr] = static_cast<uint8_t>(bcode[r] >> 8);
-                sm.st_si[mi * (kDecTileP + 16) + pr] = static_cast<uint8_t>(bcode[r] & 255u);
-            }
-        }
-        __syncthreads();
-        write_out(0);
     }
 }
 
-size_t decide_smem_bytes(const TableDev &T, const GridDev &G)
-{
-    const int nsp = (std::max(G.n_s, 1) + kDecU - 1) / kDecU * kDecU;
-    return dec_layout(T.npad, nsp, nullptr, nullptr);
-}
+size_t decide_smem_bytes(const TableDev &T, const GridDev &G) { return dec_layout(T.npad, G.n_s, nullptr, nullptr); }
 
 cudaError_t launch_decide(const DecideParams &p, cudaStream_t st)
 {

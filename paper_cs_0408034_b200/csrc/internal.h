@@ -90,10 +90,10 @@ struct DecideParams {
 
 constexpr int kDecThreads = 128;
 constexpr int kDecWarps = kDecThreads / 32;
-constexpr int kDecR = 4;                               // process counts per thread
-constexpr int kDecTileP = kDecThreads * kDecR;         // 512 process counts per CTA
-constexpr int kDecMG = 8;                              // message sizes per CTA (at most)
-constexpr int kDecU = 4;                               // candidates per filter test
+constexpr int kDecR = 8;                               // process counts per thread
+constexpr int kDecTileP = 32 * kDecR;                  // 256 process counts per CTA, shared by its warps
+constexpr int kDecMG = 16;                             // message sizes per CTA (at most), split over the warps
+constexpr int kDecU = 4;                               // list entries per filter test
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
