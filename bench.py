@@ -8,8 +8,12 @@ multi-network configuration (4096 seeded tables x P = 2..512 x 128 m x 32 s, all
 `--workload cfg3` times the exhaustive segment sweep instead.  With N > 1 every rank evaluates
 its own 4096 tables (different seeds): weak scaling, no data-path collective.
 
-Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample of
-the same workload instead (rank 0 only).
+The JSON line (ONE line, rank 0) carries the headline workload at top level and, at N = 1, a
+`workloads` list with the other configurations timed in the same run (the exhaustive sweep, the
+prediction call on the batched workload, and the three microsecond-scale configurations, marked
+launch-bound), each with its own ms_per_step, cells/s and dominant-kernel roofline object.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload instead (rank 0
+only).  Run plainly with `--gpus N` (no launcher) it starts the N ranks itself.
 """
 from __future__ import annotations
 
@@ -30,11 +34,12 @@ if ROOT not in sys.path:
 from paper_cs_0408034_b200 import workloads as wl  # noqa: E402
 
 NOMINAL_FP64_FMA_RATE = 148 * 64 * 1.965e9  # SMs x FP64 lanes per SM x max SM clock
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
-# (reduced cfg4 with 256 tables; output bytes grow in proportion to the table count, so a full launch of
-# 4096 tables is 16 x the captured one).  Set an entry to None when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_TABLE = {"decide_kernel": (163.57e6 + 0.47e6) / 256, "scatter_kernel": (159.08e6 + 0.94e6) / 256,
-                               "sweep_kernel": None}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch and per table from the ncu captures summarised
+# under profiles/ (batched workload cut to 1024 tables: 0.87 GB of output per kernel, far beyond the L2,
+# so what is still cached when the kernel ends is a few percent; traffic grows in proportion to the table
+# count).  An entry is None while its kernel has changed since the last capture.
+NCU_TRAFFIC_BYTES_PER_TABLE = {"decide_kernel": None, "scatter_kernel": None, "sweep_kernel": None}
+NCU_TRAFFIC_NOTE = "bytes per launch = bytes per table of the 1024-table ncu capture in profiles/ x tables"
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -42,6 +47,8 @@ def make_workload(name: str, scale: str, rank: int):
     if name == "cfg4":
         if scale == "small":
             return wl.config4(n_tables=256, seed_offset=1000 * rank)
+        if scale == "quarter":
+            return wl.config4(n_tables=1024, seed_offset=1000 * rank)
         return wl.config4(seed_offset=1000 * rank)
     if name == "cfg3":
         if scale == "small":
@@ -162,10 +169,28 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
-def oracle_sample_rate(w, budget_s: float):
+def _omp_set_threads(n: int) -> None:
+    """Thread count of the OpenMP runtime the oracle's shared object runs on (the oracle itself is untouched)."""
+    import ctypes
+    ctypes.CDLL("libgomp.so.1").omp_set_num_threads(int(n))
+
+
+def oracle_sample_rate(w, budget_s: float, threads: int = 0):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload: whole tables for the
-    multi-table workload, otherwise a strided subset of the process counts.  -> (cells/s, cores, text)."""
+    multi-table workload, otherwise a strided subset of the process counts.  threads = 0 keeps all host
+    cores, 1 times a single thread.  -> (cells/s, cores, text)."""
     from oracle import plogp_oracle as po
+    all_threads = po.threads()
+    if threads:
+        _omp_set_threads(threads)
+    try:
+        return _oracle_sample_rate(po, w, budget_s)
+    finally:
+        if threads:
+            _omp_set_threads(all_threads)
+
+
+def _oracle_sample_rate(po, w, budget_s: float):
     sg = po.SGrid(w.s_list) if w.s_list is not None else po.SGrid(lo=w.s_lo, hi=w.s_hi, step=w.s_step)
     per_table_cells = w.model_cells() / w.n_tables
 
@@ -197,10 +222,12 @@ def oracle_sample_rate(w, budget_s: float):
 
 
 def run_reference(args, rank):
+    """The reference arm: there is no reference implementation, so this times the CPU oracle, as it
+    stands, on a bounded sample of the workload (rank 0 only)."""
     if rank != 0:
         return
     w = make_workload(args.workload, args.scale, 0)
-    budget = 120.0 / max(1, args.steps + args.warmup)
+    budget = args.reference_budget / max(1, args.steps + args.warmup)
     rates, text, cores = [], "", 1
     for i in range(args.warmup + args.steps):
         r, cores, text = oracle_sample_rate(w, min(20.0, budget))
@@ -211,10 +238,270 @@ def run_reference(args, rank):
         "impl": "reference", "metric": "model_cells_per_sec", "value": value, "unit": "cells/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.model_cells() / value,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "call": "plogp_predict" if predict else "plogp_select_best", "note": "CPU oracle on a bounded sample; ms_per_step extrapolates to the full step"},
+        "config": {"workload": w.name, "call": "plogp_predict" if args.call == "predict" else "plogp_select_best",
+                   "note": "CPU oracle on a bounded sample; ms_per_step extrapolates to the full step"},
         "cpu_baseline": {"value": value, "unit": "cells/s", "cores": cores, "kind": "oracle", "sample": text},
         "e2e": {"value": value, "unit": "cells/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
+
+
+def predict_counts(w, counts):
+    """Work of plogp_predict on a workload: the same model cells, but every enabled plane is written out
+    (8 B per cell, plus 4 B per cell for the best segment size of each segmented strategy)."""
+    n_on = bin(w.strategy_mask).count("1")
+    n_seg = sum((w.strategy_mask >> b) & 1 for b in (2, 5, 9))
+    out_bytes = w.n_tables * w.n_P * w.n_m * (8 * n_on + 4 * n_seg)
+    slots = counts["fp64_slots"]
+    c = dict(counts)
+    if "sweep_kernel" in counts["per_kernel"]:
+        sweep = counts["per_kernel"]["sweep_kernel"]
+        c["per_kernel"] = {"sweep_kernel": sweep, "fused_kernel": {"fp64_slots": slots - sweep["fp64_slots"], "hbm_bytes": out_bytes}}
+    else:
+        c["per_kernel"] = {"fused_kernel": {"fp64_slots": slots, "hbm_bytes": out_bytes}}
+    c["hbm_bytes"] = out_bytes
+    return c
+
+
+class Bench:
+    """One rank's measuring context: device, process group, peaks."""
+
+    def __init__(self, rank, local_rank, world):
+        import torch
+        from paper_cs_0408034_b200 import plogp
+        self.torch, self.plogp = torch, plogp
+        self.rank, self.local_rank, self.world = rank, local_rank, world
+        self.dist = None
+        torch.cuda.set_device(local_rank)
+        if world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+            self.dist = dist
+        self.flush_buf = None
+        self.fma_rate = None
+        self.hbm_gbs, self.peak_src = measured_peaks()
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.destroy_process_group()
+
+    def time_device(self, w, predict, steps, warmup, clocks_uuid=None):
+        """Device-resident timing of `steps` steps of one call on one workload.  Returns the measured
+        dictionary; the per-kernel times come from events the library records around each launch."""
+        torch, plogp = self.torch, self.plogp
+        counts = work_counts(w)
+        grid = plogp.GridArgs.from_workload(w)
+        tabs = plogp.Tables.from_workload(w)
+        if predict:
+            counts = predict_counts(w, counts)
+            out = plogp.predict(tabs, grid)
+            out_bytes = counts["hbm_bytes"]
+        else:
+            out = plogp.alloc_decision(w.n_tables, w.n_P, w.n_m)
+            out_bytes = out.strategy.numel() * 13
+        flush = None
+        if out_bytes < (256 << 20):  # outputs do not evict the 126 MB L2 by themselves: write 256 MB between steps
+            if self.flush_buf is None:
+                self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+            flush = self.flush_buf
+
+        def step():
+            if predict:
+                plogp.predict(tabs, grid, out=out)
+            else:
+                plogp.select_best(tabs, grid, out=out)
+
+        for _ in range(warmup):
+            step()
+            if flush is not None:
+                flush.fill_(1)
+        self.barrier()
+        launches0 = plogp.kernel_launches()
+        plogp.profile_enable(tabs, True)
+        events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        with ClockSampler(clocks_uuid) as clocks:
+            self.barrier()
+            for a, b in events:
+                a.record()
+                step()
+                b.record()
+                if flush is not None:
+                    flush.fill_(1)
+            self.barrier()
+        launches = plogp.kernel_launches() - launches0
+        kernel_ms = plogp.profile_read(tabs)   # {kernel: (ms over the timed region, launches)}
+        plogp.profile_enable(tabs, False)
+        total_ms = max_over_ranks(sum(a.elapsed_time(b) for a, b in events), self.world, "cuda")
+        return {"w": w, "predict": predict, "counts": counts, "steps": steps, "ms_per_step": total_ms / steps, "launches": launches,
+                "kernel_ms": kernel_ms, "out_bytes": out_bytes, "flushed": flush is not None, "clocks": clocks,
+                "tabs": tabs, "grid": grid}
+
+    def time_e2e(self, m, steps):
+        """The same step through the public API with HOST buffers: the host tables go in
+        (plogp_table_update) and the decision table comes back into page-locked host arrays
+        (plogp_select_best_host); every copy is inside the timed region."""
+        plogp, w, tabs, grid = self.plogp, m["w"], m["tabs"], m["grid"]
+        host = plogp.alloc_decision_host(w.n_tables, w.n_P, w.n_m)
+        h2d = w.sizes.nbytes + w.gaps.nbytes + w.latency.nbytes + w.m.nbytes + (0 if w.s_list is None else w.s_list.nbytes)
+        d2h = sum(t.numel() * t.element_size() for t in (host.strategy, host.s_bytes, host.time))
+
+        def e2e_step():
+            tabs.update(w.sizes, w.gaps, w.latency)
+            plogp.select_best_host(tabs, grid, out=host)
+
+        e2e_step()
+        self.barrier()
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            e2e_step()
+        self.barrier()
+        ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / steps, self.world, "cuda")
+        return ms, h2d, d2h
+
+    def rooflines(self, m):
+        """Per-kernel roofline objects of one measurement, the dominant kernel's copy and the whole-step figure."""
+        if self.fma_rate is None:
+            self.fma_rate = self.plogp.fp64_fma_rate(100.0)
+        fma_rate, hbm_gbs = self.fma_rate, self.hbm_gbs
+        counts, steps, w = m["counts"], m["steps"], m["w"]
+        seg_cells = counts["segmented_cells"]
+
+        def roof(name, ms_total, n_launch):
+            # algorithmic work per launch / average launch duration (CUDA events recorded by the library on
+            # the launching stream during the timed region)
+            work = counts["per_kernel"].get(name)
+            if work is None or n_launch == 0:
+                return {"kernel": name, "launches": n_launch, "ms_total": ms_total}
+            per_launch = steps / n_launch  # a kernel launched once per step does one step's work
+            dur = ms_total / n_launch * 1e-3
+            slots, nbytes = work["fp64_slots"] * per_launch, work["hbm_bytes"] * per_launch
+            t_alu, t_hbm = slots / fma_rate, nbytes / (hbm_gbs * 1e9)
+            alu = t_alu >= t_hbm
+            r = {"kernel": name, "launches": n_launch, "ms_total": ms_total, "avg_ms": dur * 1e3,
+                 "bound": "alu" if alu else "hbm",
+                 "achieved": slots / dur / 1e12 if alu else nbytes / dur / 1e9,
+                 "peak": fma_rate / 1e12 if alu else hbm_gbs,
+                 "unit": "T FP64 thread-instr/s" if alu else "GB/s",
+                 "frac": max(t_alu, t_hbm) / dur,
+                 "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
+                 "peak_source": ("DFMA issue rate measured in this run by plogp_fp64_fma_rate, of measured (nominal %.2f T/s = 148 SMs x 64 lanes x 1.965 GHz)"
+                                 % (NOMINAL_FP64_FMA_RATE / 1e12)) if alu else "HBM copy bandwidth, of %s" % self.peak_src}
+            if alu and name in ("sweep_kernel", "decide_kernel"):
+                # stricter accounting: the compare of a segmented cell runs in the integer pipe, so only its DFMA
+                # is an FP64 slot (1 instead of 2 per segmented cell)
+                strict = (work["fp64_slots"] - seg_cells) * per_launch
+                r["frac_dfma_only"] = max(strict / fma_rate, t_hbm) / dur
+            return r
+
+        kernels = [roof(k, v[0], v[1]) for k, v in m["kernel_ms"].items()]
+        tot = sum(k["ms_total"] for k in kernels) or 1.0
+        for k in kernels:
+            k["share"] = k["ms_total"] / tot
+        dominant = dict(max(kernels, key=lambda k: k["ms_total"])) if kernels else {}
+        per_table = NCU_TRAFFIC_BYTES_PER_TABLE.get(dominant.get("kernel"))
+        batched = w.name.startswith("cfg4") and not m["predict"]
+        dominant["traffic"] = per_table * w.n_tables if (per_table and batched) else None
+        dominant["traffic_note"] = NCU_TRAFFIC_NOTE if dominant["traffic"] else None
+        t_alu = counts["fp64_slots"] / fma_rate
+        t_hbm = counts["hbm_bytes"] / (hbm_gbs * 1e9)
+        dominant["step"] = {"frac": max(t_alu, t_hbm) / (m["ms_per_step"] * 1e-3), "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
+                            "note": "whole step (all kernels) against max(FP64 issue, HBM bytes)"}
+        return kernels, dominant
+
+    def config_of(self, m):
+        w, counts = m["w"], m["counts"]
+        return {"workload": w.name, "call": "plogp_predict" if m["predict"] else "plogp_select_best", "tables_per_gpu": w.n_tables,
+                "P": [w.P_lo, w.P_hi], "n_m": w.n_m, "n_s": int(len(w.s_values())), "strategy_mask": w.strategy_mask,
+                "model_cells_per_gpu": counts["model_cells"], "decision_cells_per_gpu": counts["decision_cells"],
+                "parallelism": "tables sharded, %d rank(s)" % self.world,
+                "l2": "256 MB written between timed steps to flush L2" if m["flushed"]
+                else "outputs (%.1f GB per step) exceed the 126 MB L2" % (m["out_bytes"] / 1e9)}
+
+    def entry(self, m, note=None):
+        """One element of the `workloads` list."""
+        kernels, dominant = self.rooflines(m)
+        step_s = m["ms_per_step"] * 1e-3
+        e = {"config": self.config_of(m), "steps": m["steps"], "ms_per_step": m["ms_per_step"],
+             "model_cells_per_sec": m["counts"]["model_cells"] / step_s, "decision_cells_per_sec": m["counts"]["decision_cells"] / step_s,
+             "gpu_launches_per_step": m["launches"] / m["steps"], "roofline": dominant}
+        if note:
+            e["note"] = note
+        return e
+
+
+def _free(m):
+    m["tabs"].free()
+    m.pop("tabs"); m.pop("grid")
+
+
+def run_ours(args, rank, local_rank, world):
+    if args.warmup < 3:
+        args.warmup = 3
+    b = Bench(rank, local_rank, world)
+    torch = b.torch
+    uuid = str(torch.cuda.get_device_properties(local_rank).uuid)
+    if not uuid.startswith("GPU-"):
+        uuid = "GPU-" + uuid
+
+    w = make_workload(args.workload, args.scale, rank)
+    predict = args.call == "predict"
+    m = b.time_device(w, predict, args.steps, args.warmup, clocks_uuid=uuid)
+    e2e_ms, h2d, d2h = None, 0, 0
+    if args.e2e_steps > 0 and not predict:
+        e2e_ms, h2d, d2h = b.time_e2e(m, args.e2e_steps)
+    _free(m)
+    if rank != 0:
+        b.close()
+        return
+
+    kernels, roofline = b.rooflines(m)
+    counts, step_s = m["counts"], m["ms_per_step"] * 1e-3
+    line = {
+        "metric": "model_cells_per_sec", "value": world * counts["model_cells"] / step_s, "unit": "cells/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": m["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "decision_cells_per_sec": world * counts["decision_cells"] / step_s,
+        "config": b.config_of(m),
+        "clocks": m["clocks"].summary(),
+        "e2e": {"value": None if e2e_ms is None else world * counts["model_cells"] / (e2e_ms * 1e-3), "unit": "cells/s",
+                "ms_per_step": e2e_ms, "steps": args.e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": m["launches"],
+        "roofline": roofline,
+        "kernels": kernels,
+    }
+    if world == 1 and not args.no_workloads and args.workload == "cfg4" and args.scale == "full" and not predict:
+        # the other configurations, in the same run: fewer steps, same timing rules
+        others = []
+        k = max(3, min(args.steps, 10))
+        mm = b.time_device(wl.config3(), False, k, 3)
+        _free(mm)
+        others.append(b.entry(mm))
+        mm = b.time_device(w, True, k, 3)
+        _free(mm)
+        others.append(b.entry(mm))
+        for make in (wl.config2, wl.config5, wl.config1):
+            mm = b.time_device(make(), False, max(k, 20), 5)
+            _free(mm)
+            others.append(b.entry(mm, note="launch-bound: microseconds of work per call; reported, not judged against the 60 % bar"))
+        line["workloads"] = others
+    if world == 1 and not args.no_cpu_baseline:
+        v, cores, text = oracle_sample_rate(w, 15.0)
+        v1, _, text1 = oracle_sample_rate(w, 8.0, threads=1)
+        line["cpu_baseline"] = {"value": v, "unit": "cells/s", "cores": cores, "kind": "oracle", "sample": text,
+                                "single_thread": {"value": v1, "unit": "cells/s", "cores": 1, "sample": text1}}
+    print(json.dumps(line))
+    b.close()
+
+
+def _spawned(local_rank, argv, world, port):
+    os.environ.update(RANK=str(local_rank), LOCAL_RANK=str(local_rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    sys.argv = argv
+    main()
 
 
 def main():
@@ -224,185 +511,31 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
-    ap.add_argument("--scale", default="full", choices=["full", "small"], help="small: reduced copy for profiler captures")
+    ap.add_argument("--scale", default="full", choices=["full", "quarter", "small"],
+                    help="quarter / small: reduced copies of the batched workload and the sweep for profiler captures")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--call", default="select_best", choices=["select_best", "predict"],
                     help="predict: time plogp_predict (all model planes) instead of the decision table; device-resident only")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true", help="headline workload only (no `workloads` list)")
+    ap.add_argument("--reference-budget", type=float, default=120.0, help="seconds of oracle time for --impl reference")
     args = ap.parse_args()
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
-        run_reference(args, rank)
+        run_reference(args, int(os.environ.get("RANK", "0")))
         return
-    if args.warmup < 3:
-        args.warmup = 3
-
-    import torch
-    import torch.distributed as dist
-    from paper_cs_0408034_b200 import plogp
-
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    w = make_workload(args.workload, args.scale, rank)
-    counts = work_counts(w)
-    grid = plogp.GridArgs.from_workload(w)
-    tabs = plogp.Tables.from_workload(w)
-    predict = args.call == "predict"
-    if predict:
-        # all enabled model planes (8 B) plus the best segment size of each segmented strategy (4 B)
-        out = plogp.predict(tabs, grid)
-        torch.cuda.synchronize()
-        n_on = bin(w.strategy_mask).count("1")
-        n_seg = sum((w.strategy_mask >> b) & 1 for b in (2, 5, 9))
-        out_bytes = w.n_tables * w.n_P * w.n_m * (8 * n_on + 4 * n_seg)
-        slots = counts["fp64_slots"]
-        if "sweep_kernel" in counts["per_kernel"]:
-            counts["per_kernel"] = {"sweep_kernel": counts["per_kernel"]["sweep_kernel"],
-                                    "fused_kernel": {"fp64_slots": slots - counts["per_kernel"]["sweep_kernel"]["fp64_slots"], "hbm_bytes": out_bytes}}
-        else:
-            counts["per_kernel"] = {"fused_kernel": {"fp64_slots": slots, "hbm_bytes": out_bytes}}
-        counts["hbm_bytes"] = out_bytes
-        args.e2e_steps = 0
-    else:
-        out = plogp.alloc_decision(w.n_tables, w.n_P, w.n_m)
-        out_bytes = out.strategy.numel() * 13
-    flush = None
-    if out_bytes < (256 << 20):  # outputs do not evict the 126 MB L2 by themselves: write 256 MB between steps
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-
-    def step():
-        if predict:
-            plogp.predict(tabs, grid, out=out)
-        else:
-            plogp.select_best(tabs, grid, out=out)
-
-    for _ in range(args.warmup):
-        step()
-        if flush is not None:
-            flush.fill_(1)
-    barrier()
-
-    uuid = str(torch.cuda.get_device_properties(local_rank).uuid)
-    if not uuid.startswith("GPU-"):
-        uuid = "GPU-" + uuid
-    launches0 = plogp.kernel_launches()
-    plogp.profile_enable(tabs, True)
-    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    with ClockSampler(uuid) as clocks:
-        barrier()
-        for a, b in events:
-            a.record()
-            step()
-            b.record()
-            if flush is not None:
-                flush.fill_(1)
-        barrier()
-    launches = plogp.kernel_launches() - launches0
-    kernel_ms = plogp.profile_read(tabs)   # {kernel: (ms over the timed region, launches)}
-    plogp.profile_enable(tabs, False)
-    total_ms = sum(a.elapsed_time(b) for a, b in events)
-    total_ms = max_over_ranks(total_ms, world, "cuda")
-    ms_per_step = total_ms / args.steps
-
-    # ---- end to end through the public API with host buffers ----
-    e2e_ms, h2d, d2h = None, 0, 0
-    if args.e2e_steps > 0:
-        host = plogp.alloc_decision_host(w.n_tables, w.n_P, w.n_m)   # page-locked
-        h2d = w.sizes.nbytes + w.gaps.nbytes + w.latency.nbytes + w.m.nbytes + (0 if w.s_list is None else w.s_list.nbytes)
-        d2h = sum(t.numel() * t.element_size() for t in (host.strategy, host.s_bytes, host.time))
-
-        def e2e_step():
-            # host arrays in (plogp_table_update), host arrays out (plogp_select_best_host): every copy is inside
-            tabs.update(w.sizes, w.gaps, w.latency)
-            plogp.select_best_host(tabs, grid, out=host)
-
-        e2e_step()
-        barrier()
-        t0 = time.perf_counter()
-        for _ in range(args.e2e_steps):
-            e2e_step()
-        barrier()
-        e2e_ms = (time.perf_counter() - t0) * 1e3 / args.e2e_steps
-        e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
-        del host
-
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        # started without a launcher: one process per GPU from here
+        import socket
+        import torch.multiprocessing as mp
+        s = socket.socket()
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+        s.close()
+        mp.spawn(_spawned, args=(list(sys.argv), args.gpus, port), nprocs=args.gpus, join=True)
         return
-
-    fma_rate = plogp.fp64_fma_rate(100.0)
-    hbm_gbs, peak_src = measured_peaks()
-    step_s = ms_per_step * 1e-3
-
-    def roof(name, ms_total, n_launch):
-        """Roofline of one kernel: algorithmic work per launch / its average launch duration (CUDA events
-        recorded by the library on the launching stream during the timed region)."""
-        work = counts["per_kernel"].get(name)
-        if work is None or n_launch == 0:
-            return {"kernel": name, "launches": n_launch, "ms_total": ms_total}
-        per_launch = args.steps / n_launch  # a kernel launched once per step does one step's work
-        dur = ms_total / n_launch * 1e-3
-        slots, nbytes = work["fp64_slots"] * per_launch, work["hbm_bytes"] * per_launch
-        t_alu, t_hbm = slots / fma_rate, nbytes / (hbm_gbs * 1e9)
-        alu = t_alu >= t_hbm
-        return {"kernel": name, "launches": n_launch, "ms_total": ms_total, "avg_ms": dur * 1e3,
-                "bound": "alu" if alu else "hbm",
-                "achieved": slots / dur / 1e12 if alu else nbytes / dur / 1e9,
-                "peak": fma_rate / 1e12 if alu else hbm_gbs,
-                "unit": "T FP64 thread-instr/s" if alu else "GB/s",
-                "frac": max(t_alu, t_hbm) / dur,
-                "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
-                "peak_source": ("DFMA issue rate measured in this run by plogp_fp64_fma_rate, of measured (nominal %.2f T/s = 148 SMs x 64 lanes x 1.965 GHz)"
-                                % (NOMINAL_FP64_FMA_RATE / 1e12)) if alu else "HBM copy bandwidth, of %s" % peak_src}
-
-    kernels = [roof(k, v[0], v[1]) for k, v in kernel_ms.items()]
-    tot_kernel_ms = sum(k["ms_total"] for k in kernels) or 1.0
-    for k in kernels:
-        k["share"] = k["ms_total"] / tot_kernel_ms
-    dominant = max(kernels, key=lambda k: k["ms_total"]) if kernels else {}
-    roofline = dict(dominant)
-    per_table = NCU_TRAFFIC_BYTES_PER_TABLE.get(dominant.get("kernel"))
-    roofline["traffic"] = per_table * w.n_tables if (per_table and args.workload == "cfg4") else None
-    roofline["traffic_note"] = "bytes per launch, scaled from the 256-table ncu capture in profiles/" if roofline["traffic"] else None
-    t_alu = counts["fp64_slots"] / fma_rate
-    t_hbm = counts["hbm_bytes"] / (hbm_gbs * 1e9)
-    roofline["step"] = {"frac": max(t_alu, t_hbm) / step_s, "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
-                        "note": "whole step (all kernels) against max(FP64 issue, HBM bytes)"}
-
-    line = {
-        "metric": "model_cells_per_sec", "value": world * counts["model_cells"] / step_s, "unit": "cells/s",
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "decision_cells_per_sec": world * counts["decision_cells"] / step_s,
-        "config": {"workload": w.name, "call": "plogp_predict" if predict else "plogp_select_best", "tables_per_gpu": w.n_tables, "P": [w.P_lo, w.P_hi], "n_m": w.n_m,
-                   "n_s": int(len(w.s_values())), "strategy_mask": w.strategy_mask, "model_cells_per_gpu": counts["model_cells"],
-                   "decision_cells_per_gpu": counts["decision_cells"], "parallelism": "tables sharded, %d rank(s)" % world,
-                   "l2": ("outputs (%.1f GB per step) exceed the 126 MB L2" % (out_bytes / 1e9)) if flush is None
-                   else "256 MB written between timed steps to flush L2"},
-        "clocks": clocks.summary(),
-        "e2e": {"value": None if e2e_ms is None else world * counts["model_cells"] / (e2e_ms * 1e-3), "unit": "cells/s",
-                "ms_per_step": e2e_ms, "steps": args.e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": launches,
-        "roofline": roofline,
-        "kernels": kernels,
-    }
-    if world == 1 and not args.no_cpu_baseline:
-        v, cores, text = oracle_sample_rate(w, 15.0)
-        line["cpu_baseline"] = {"value": v, "unit": "cells/s", "cores": cores, "kind": "oracle", "sample": text}
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    run_ours(args, int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+             int(os.environ.get("WORLD_SIZE", "1")))
 
 
 if __name__ == "__main__":

@@ -172,7 +172,7 @@ class GridArgs:
 
     @classmethod
     def from_workload(cls, w) -> "GridArgs":
-        return cls(w.m, None, w.P_lo, w.P_hi, w.s_list, w.s_lo, w.s_hi, w.s_step, w.dtype_bytes,
+        return cls(w.m, getattr(w, "P_list", None), w.P_lo, w.P_hi, w.s_list, w.s_lo, w.s_hi, w.s_step, w.dtype_bytes,
                    w.strategy_mask, w.k_mode)
 
     @property

@@ -82,6 +82,7 @@ class Workload:
     dtype_bytes: int = 4
     seed: int = 0
     notes: dict = field(default_factory=dict)
+    P_list: Optional[np.ndarray] = None   # int32 ascending process counts; None => P_lo..P_hi
 
     @property
     def n_tables(self) -> int:
@@ -97,13 +98,15 @@ class Workload:
 
     @property
     def n_P(self) -> int:
-        return self.P_hi - self.P_lo + 1
+        return len(self.P_list) if self.P_list is not None else self.P_hi - self.P_lo + 1
 
     @property
     def n_m(self) -> int:
         return len(self.m)
 
     def P_values(self) -> np.ndarray:
+        if self.P_list is not None:
+            return np.asarray(self.P_list, dtype=np.int64)
         return np.arange(self.P_lo, self.P_hi + 1, dtype=np.int64)
 
     def s_values(self) -> np.ndarray:

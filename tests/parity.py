@@ -143,3 +143,49 @@ def check_decision(w, ot, dec, tables=None, p_idx=None, m_idx=None) -> int:
                 assert (alt - best) / best <= TIE_MARGIN, (where, alt, best)
             n += g_id[c].size
     return n
+
+
+def check_decision_cells(w, dec, t_idx, p_idx, m_idx, table_cache=None) -> int:
+    """Decision cells given one by one (table, P index, m index), each re-decided by the oracle on its
+    own (po.decide: every enabled strategy, exhaustive segment search) — for launch shapes whose whole
+    tables the oracle cannot redo.  Both collectives of every sampled cell are checked."""
+    import torch
+    t_idx, p_idx, m_idx = (np.asarray(x, dtype=np.int64) for x in (t_idx, p_idx, m_idx))
+    dev = dec.strategy.device
+    ti, pi, mi = (torch.as_tensor(x, device=dev) for x in (t_idx, p_idx, m_idx))
+    g_id = dec.strategy[ti, :, pi, mi].cpu().numpy()
+    g_s = dec.s_bytes[ti, :, pi, mi].cpu().numpy().view(np.uint32)
+    g_t = dec.time[ti, :, pi, mi].cpu().numpy()
+    sg = oracle_sgrid(w)
+    mask = w.strategy_mask
+    Ps = w.P_values()
+    cache = {} if table_cache is None else table_cache
+    n = 0
+    for i in range(len(t_idx)):
+        t = int(t_idx[i])
+        if t not in cache:
+            cache[t] = po.Table(w.table_sizes(t), w.gaps[t], w.latency[t])
+        tab = cache[t]
+        P, m = int(Ps[p_idx[i]]), int(w.m[m_idx[i]])
+        for c, bits in ((0, mask & 0x3FF), (1, mask & 0x1C00)):
+            if not bits:
+                continue
+            sid, s, best, _ = po.decide(tab, c, mask, P, m, sg, w.k_mode)
+            gid, gs, gt = int(g_id[i, c]), int(g_s[i, c]), float(g_t[i, c])
+            where = "table %d coll %d P %d m %d" % (t, c, P, m)
+            n += 1
+            if gid == sid and gs == s:
+                assert _rel(gt, best) <= TIME_RTOL, (where, gt, best)
+                continue
+            # another pick: only inside the tie margin, and with the oracle's time for that very pick
+            assert (mask >> gid) & 1 and (gid < 10) == (c == 0), "%s: strategy %d not eligible" % (where, gid)
+            if gid in SEG_IDS:
+                assert _valid_s(w, m, gs), "%s: %d is not a candidate segment size" % (where, gs)
+                alt = po.model(tab, gid, P, m, gs, w.k_mode)
+            else:
+                assert gs == 0, where
+                alt = po.model(tab, gid, P, m, 0, w.k_mode)
+            assert (alt - best) / best <= TIE_MARGIN, "%s: picked (%d, %d) at %.17g, oracle (%d, %d) at %.17g" % (
+                where, gid, gs, alt, sid, s, best)
+            assert _rel(gt, alt) <= TIME_RTOL, (where, gt, alt)
+    return n
