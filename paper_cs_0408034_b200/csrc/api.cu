@@ -417,6 +417,8 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             dp.n_mgroups = pl.dec_mgroups; dp.n_ptiles = pl.dec_ptiles; dp.mg = pl.dec_mg;
             dp.table0 = t0; dp.n_tables_launch = nt;
             dp.d_strategy = out.d_strategy; dp.d_sbytes = out.d_sbytes; dp.d_time = out.d_time;
+            dp.vec_out = (pl.G.n_m % 2 == 0) && pl.dec_mg >= 2 && reinterpret_cast<uintptr_t>(out.d_time) % 16 == 0 &&
+                         reinterpret_cast<uintptr_t>(out.d_sbytes) % 8 == 0 && reinterpret_cast<uintptr_t>(out.d_strategy) % 2 == 0;
             { LaunchTimer lt(h, PLOGP_KERNEL_DECIDE, st); CK(launch_decide(dp, st)); }
             g_launches += 1;
             Gf.mask &= 0x1C00u;

@@ -41,9 +41,10 @@ constexpr uint32_t kCandNone = 255;   // winner is an unsegmented strategy
 constexpr uint32_t kCandWhole = 254;  // segmented winner with no fitting candidate: the whole message
 constexpr uint32_t kCodeNever = 0xFFFFu;
 constexpr unsigned kNoPilot = 0x1FFu;
+constexpr int kIntMax = 0x7FFFFFFF;
 
 struct DecSmem {
-    double *tab, *gs, *gm, *lf, *lc, *l2, *st_time;
+    double *tab, *gs, *gm, *lf, *lc, *pm1, *l2, *st_time;
     double2 *l1;
     uint32_t *sval;
     uint16_t *c1, *c2, *st_code;
@@ -60,7 +61,7 @@ __host__ __device__ inline size_t dec_layout(int npad, int n_s, unsigned char *b
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off += (bytes + 15) & ~size_t(15); return at; };
     const size_t o_tab = take(3 * size_t(npad) * 8), o_gs = take(size_t(nsv) * 8), o_sv = take(size_t(nsv) * 4),
-                 o_gm = take(kDecMG * 8), o_lf = take(kDecTileP * 8), o_lc = take(kDecTileP * 8),
+                 o_gm = take(kDecMG * 8), o_lf = take(kDecTileP * 8), o_lc = take(kDecTileP * 8), o_pm = take(kDecTileP * 8),
                  o_l1 = take(size_t(kDecWarps) * cap1 * 16), o_l2 = take(size_t(kDecWarps) * cap2 * 8),
                  o_c1 = take(size_t(kDecWarps) * cap1 * 2), o_c2 = take(size_t(kDecWarps) * cap2 * 2),
                  o_t = take(size_t(kDecMG) * kStageStride * 8), o_c = take(size_t(kDecMG) * kCodeStride * 2);
@@ -68,6 +69,7 @@ __host__ __device__ inline size_t dec_layout(int npad, int n_s, unsigned char *b
         o->tab = reinterpret_cast<double *>(base + o_tab); o->gs = reinterpret_cast<double *>(base + o_gs);
         o->sval = reinterpret_cast<uint32_t *>(base + o_sv); o->gm = reinterpret_cast<double *>(base + o_gm);
         o->lf = reinterpret_cast<double *>(base + o_lf); o->lc = reinterpret_cast<double *>(base + o_lc);
+        o->pm1 = reinterpret_cast<double *>(base + o_pm);
         o->l1 = reinterpret_cast<double2 *>(base + o_l1); o->l2 = reinterpret_cast<double *>(base + o_l2);
         o->c1 = reinterpret_cast<uint16_t *>(base + o_c1); o->c2 = reinterpret_cast<uint16_t *>(base + o_c2);
         o->st_time = reinterpret_cast<double *>(base + o_t); o->st_code = reinterpret_cast<uint16_t *>(base + o_c);
@@ -77,6 +79,15 @@ __host__ __device__ inline size_t dec_layout(int npad, int n_s, unsigned char *b
 }
 
 __device__ __forceinline__ int hi32(double x) { return __double2hiint(x); }
+
+// Exact comparison of one cell with the running minimum: (time, code) in lexicographic order, where the code
+// orders strategy id first and candidate index (= segment size order) second.
+__device__ __forceinline__ void offer(double &bt, uint32_t &bcode, double t, uint32_t code)
+{
+    if (t <= bt) {
+        if (t < bt || code < bcode) { bt = t; bcode = code; }
+    }
+}
 
 }  // namespace
 
@@ -106,6 +117,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
         const int P = P_at(p.G, min(tile0 + i, p.G.n_P - 1));
         sm.lf[i] = static_cast<double>(31 - __clz(P));
         sm.lc[i] = static_cast<double>(32 - __clz(P - 1));
+        sm.pm1[i] = static_cast<double>(P - 1);
     }
     __syncthreads();
     const double L = p.T.lat[table];
@@ -122,10 +134,8 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     const double rdv = 2.0 * g1 + 3.0 * L;  // rendezvous handshake: 2 g(1) + 3 L
     __syncthreads();
 
-    // this thread's cells: process counts at tile offset 32 r + lane
-    double pm1[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) pm1[r] = static_cast<double>(P_at(p.G, min(tile0 + 32 * r + lane, p.G.n_P - 1)) - 1);
+    // this thread's cells: process counts at tile offset 32 r + lane; P-1, floor(log2 P) and ceil(log2 P) are read
+    // from shared memory where a loop needs them, so that only one of the sets is live at a time
     // the pilot's process count: middle of the tile's valid range
     const int P_mid = P_at(p.G, tile0 + n_valid / 2);
     const double x1_mid = static_cast<double>(P_mid - 1);
@@ -154,7 +164,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
         __syncwarp();  // the previous message size's loops have finished reading the lists
         double tb = CUDART_INF;
         unsigned pb = kNoPilot;  // P-list position, or 256 + log-list position
-        auto offer = [&](double t, unsigned pos) {
+        auto pilot_offer = [&](double t, unsigned pos) {
             if (t < tb) { tb = t; pb = pos; }
         };
         if (lane < 4) {
@@ -166,13 +176,13 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 const double c = id >= 3 ? 0.0 : (id == 1 ? rdv : L);
                 l1[pos] = make_double2(a, c);
                 c1[pos] = static_cast<uint16_t>((id << 8) | kCandNone);
-                offer(fma(x1_mid, a, c), pos);
+                pilot_offer(fma(x1_mid, a, c), pos);
             }
         }
         if (lane == 4 && has7) {  // Binomial Tree
             l2[0] = gm;
             c2[0] = static_cast<uint16_t>((7u << 8) | kCandNone);
-            offer(fma(x2_mid, gm, c2_mid), 256u);
+            pilot_offer(fma(x2_mid, gm, c2_mid), 256u);
         }
         for (int i = n1 + lane; i < n1p; i += 32) {  // padding never reaches the minimum
             l1[i] = make_double2(CUDART_INF, CUDART_INF);
@@ -195,18 +205,18 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             if (has2) {  // (P-1) (g(s) k) + L
                 l1[o2 + c] = make_double2(Q, L);
                 c1[o2 + c] = static_cast<uint16_t>((2u << 8) | cand);
-                offer(fma(x1_mid, Q, L), o2 + c);
+                pilot_offer(fma(x1_mid, Q, L), o2 + c);
             }
             if (has5) {  // (P-1) (g(s) + L) + g(s) (k-1)
                 const double B = gsv + L, C = gsv * (k - 1.0);
                 l1[o5 + c] = make_double2(B, C);
                 c1[o5 + c] = static_cast<uint16_t>((5u << 8) | cand);
-                offer(fma(x1_mid, B, C), o5 + c);
+                pilot_offer(fma(x1_mid, B, C), o5 + c);
             }
             if (has9) {  // floor(log2 P) g(s) k + ceil(log2 P) L
                 l2[o9 + c] = Q;
                 c2[o9 + c] = static_cast<uint16_t>((9u << 8) | cand);
-                offer(fma(x2_mid, Q, c2_mid), 256u + o9 + c);
+                pilot_offer(fma(x2_mid, Q, c2_mid), 256u + o9 + c);
             }
         }
         // warp-wide pilot: smallest time (high word first, then low word with the position in its last 9 bits)
@@ -234,7 +244,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             __syncwarp();
             if (lane == 0) l1[pilot] = make_double2(CUDART_INF, CUDART_INF);
 #pragma unroll
-            for (int r = 0; r < R; ++r) { bt[r] = fma(pm1[r], e.x, e.y); bcode[r] = code; }
+            for (int r = 0; r < R; ++r) { bt[r] = fma(sm.pm1[32 * r + lane], e.x, e.y); bcode[r] = code; }
         } else {
             const double a = l2[pilot - 256u];
             const uint32_t code = c2[pilot - 256u];
@@ -247,13 +257,13 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
 
         // one cell per process count (ids 6 and 8): high-word test, exact comparison where it holds
         auto single = [&](uint32_t code, const double *t) {
-            bool f[R], any = false;
+            int acc = kIntMax;
 #pragma unroll
-            for (int r = 0; r < R; ++r) { f[r] = hi32(t[r]) <= hi32(bt[r]); any |= f[r]; }
-            if (any) {
+            for (int r = 0; r < R; ++r) acc = min(acc, hi32(t[r]) - hi32(bt[r]));
+            if (acc <= 0) {
 #pragma unroll
                 for (int r = 0; r < R; ++r)
-                    if (f[r] && (t[r] < bt[r] || (t[r] == bt[r] && code < bcode[r]))) { bt[r] = t[r]; bcode[r] = code; }
+                    if (t[r] < bt[r] || (t[r] == bt[r] && code < bcode[r])) { bt[r] = t[r]; bcode[r] = code; }
             }
         };
         if (has6) {  // Binary Tree (the printed bound): ceil(log2 P) (2 g(m) + L)
@@ -272,55 +282,61 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
 #pragma unroll
         for (int r = 0; r < R; ++r) lcL[r] *= L;
 
+        // The filter of a group of U list entries: every cell is evaluated (one DFMA each); per process
+        // count the smallest high word of the U times minus the high word of the running minimum says
+        // whether a cell can reach it (<= 0), and the differences of all R process counts are folded into
+        // one minimum, so the test costs integer min / add instructions only (no predicates, no branches)
+        // and a single vote decides whether the group needs the exact pass.  The exact pass, (time, id,
+        // candidate) in lexicographic order, runs for the rows r that some lane flagged.
+
         // ---- log list: t = fma(floor(log2 P), a, ceil(log2 P) L) ----
 #pragma unroll 1
         for (int j = 0; j < n2p; j += U) {
             const double2 q01 = *reinterpret_cast<const double2 *>(l2 + j), q23 = *reinterpret_cast<const double2 *>(l2 + j + 2);
-            bool f[R], any = false;
+            int acc = kIntMax;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const int h0 = hi32(fma(lf[r], q01.x, lcL[r])), h1 = hi32(fma(lf[r], q01.y, lcL[r]));
                 const int h2 = hi32(fma(lf[r], q23.x, lcL[r])), h3 = hi32(fma(lf[r], q23.y, lcL[r]));
-                f[r] = min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]);
-                any |= f[r];
+                acc = min(acc, min(min(h0, h1), min(h2, h3)) - hi32(bt[r]));
             }
-            if (__any_sync(kFull, any)) {  // rare: exact comparison, (time, id, candidate) in lexicographic order
+            if (__any_sync(kFull, acc <= 0)) {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    if (__any_sync(kFull, f[r])) {
+                    const int h0 = hi32(fma(lf[r], q01.x, lcL[r])), h1 = hi32(fma(lf[r], q01.y, lcL[r]));
+                    const int h2 = hi32(fma(lf[r], q23.x, lcL[r])), h3 = hi32(fma(lf[r], q23.y, lcL[r]));
+                    if (__any_sync(kFull, min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]))) {
 #pragma unroll 1
-                        for (int u = 0; u < U; ++u) {
-                            const double t = fma(lf[r], l2[j + u], lcL[r]);
-                            const uint32_t code = c2[j + u];
-                            if (t < bt[r] || (t == bt[r] && code < bcode[r])) { bt[r] = t; bcode[r] = code; }
-                        }
+                        for (int u = 0; u < U; ++u) offer(bt[r], bcode[r], fma(lf[r], l2[j + u], lcL[r]), c2[j + u]);
                     }
                 }
             }
         }
 
         // ---- P list: t = fma(P-1, a, c) ----
+        double pm1[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) pm1[r] = sm.pm1[32 * r + lane];
 #pragma unroll 1
         for (int j = 0; j < n1p; j += U) {
             const double2 e0 = l1[j], e1 = l1[j + 1], e2 = l1[j + 2], e3 = l1[j + 3];
-            bool f[R], any = false;
+            int acc = kIntMax;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const int h0 = hi32(fma(pm1[r], e0.x, e0.y)), h1 = hi32(fma(pm1[r], e1.x, e1.y));
                 const int h2 = hi32(fma(pm1[r], e2.x, e2.y)), h3 = hi32(fma(pm1[r], e3.x, e3.y));
-                f[r] = min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]);
-                any |= f[r];
+                acc = min(acc, min(min(h0, h1), min(h2, h3)) - hi32(bt[r]));
             }
-            if (__any_sync(kFull, any)) {
+            if (__any_sync(kFull, acc <= 0)) {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    if (__any_sync(kFull, f[r])) {
+                    const int h0 = hi32(fma(pm1[r], e0.x, e0.y)), h1 = hi32(fma(pm1[r], e1.x, e1.y));
+                    const int h2 = hi32(fma(pm1[r], e2.x, e2.y)), h3 = hi32(fma(pm1[r], e3.x, e3.y));
+                    if (__any_sync(kFull, min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]))) {
 #pragma unroll 1
                         for (int u = 0; u < U; ++u) {
                             const double2 e = l1[j + u];
-                            const double t = fma(pm1[r], e.x, e.y);
-                            const uint32_t code = c1[j + u];
-                            if (t < bt[r] || (t == bt[r] && code < bcode[r])) { bt[r] = t; bcode[r] = code; }
+                            offer(bt[r], bcode[r], fma(pm1[r], e.x, e.y), c1[j + u]);
                         }
                     }
                 }
@@ -336,7 +352,28 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     __syncthreads();
 
     // transposed write-out of the staged group: rows of p.mg consecutive m per process count
-    {
+    if (p.vec_out) {
+        // two message sizes per lane: 16-byte, 8-byte and 2-byte stores (the host has checked the alignment)
+        const int half = p.mg >> 1;
+        const int mi = 2 * (lane & (half - 1)), prow = lane / half, rows = 32 / half;
+        if (mi < n_mi) {
+            const uint32_t m_u0 = p.G.m_list[m0 + mi], m_u1 = p.G.m_list[m0 + mi + 1];
+            const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
+            const size_t base = static_cast<size_t>(table) * 2 * plane + static_cast<size_t>(m0 + mi);
+            const double *st0 = sm.st_time + mi * kStageStride, *st1 = st0 + kStageStride;
+            const uint16_t *sc0 = sm.st_code + mi * kCodeStride, *sc1 = sc0 + kCodeStride;
+            for (int pr = warp * rows + prow; pr < n_valid; pr += kDecWarps * rows) {
+                const size_t o = base + static_cast<size_t>(tile0 + pr) * p.G.n_m;
+                const uint32_t code0 = sc0[pr], code1 = sc1[pr];
+                const uint32_t cand0 = code0 & 255u, cand1 = code1 & 255u;
+                const uint32_t s0 = cand0 == kCandNone ? 0u : (cand0 == kCandWhole ? m_u0 : sm.sval[cand0]);
+                const uint32_t s1 = cand1 == kCandNone ? 0u : (cand1 == kCandWhole ? m_u1 : sm.sval[cand1]);
+                *reinterpret_cast<double2 *>(p.d_time + o) = make_double2(st0[pr], st1[pr]);
+                *reinterpret_cast<uint2 *>(p.d_sbytes + o) = make_uint2(s0, s1);
+                *reinterpret_cast<uint16_t *>(p.d_strategy + o) = static_cast<uint16_t>((code0 >> 8) | (code1 & 0xFF00u));
+            }
+        }
+    } else {
         const int mi = lane & (p.mg - 1), prow = lane / p.mg, rows = 32 / p.mg;
         if (mi < n_mi) {
             const uint32_t m_u = p.G.m_list[m0 + mi];

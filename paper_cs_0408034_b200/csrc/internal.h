@@ -82,6 +82,7 @@ struct DecideParams {
     GridDev G;
     int n_mgroups, n_ptiles;
     int mg;  // message sizes per CTA, 1..kDecMG
+    int vec_out;  // outputs aligned for two message sizes per store (n_m even, 16 / 8 / 2-byte aligned bases)
     int table0, n_tables_launch;
     uint8_t *d_strategy;
     uint32_t *d_sbytes;
