@@ -61,7 +61,9 @@ typedef enum {
     PLOGP_E_NOMEM = -2, /* host or device allocation failed */
     PLOGP_E_CUDA = -3,  /* a CUDA runtime call failed; plogp_last_cuda_error() names it */
     PLOGP_E_RANGE = -4  /* m, s or a table size too large: m and s must be < 2^32, sizes < 2^53,
-                           n_bp <= PLOGP_MAX_BREAKPOINTS, P_hi * m < 2^53 (so that j * m is exact in a double) */
+                           n_bp <= PLOGP_MAX_BREAKPOINTS, P <= 2^30, P_hi * m < 2^53 (so that j * m is exact in a
+                           double); or a table whose last gap is below the one before it (continued above the
+                           table, that line would make g negative) */
 } plogp_status;
 
 /* Opaque set of pLogP parameter tables resident on the current CUDA device. */
@@ -71,7 +73,8 @@ typedef struct plogp_tables plogp_tables;
  * Upload n_tables independent pLogP parameter sets (Section 2: gap g at n_bp message sizes and
  * the latency L of each network).
  *   sizes_bytes  HOST, [n_bp] when sizes_shared != 0, else [n_tables][n_bp]; strictly increasing.
- *   gap          HOST, [n_tables][n_bp]; finite, >= 0; any time unit (the outputs use the same).
+ *   gap          HOST, [n_tables][n_bp]; finite, >= 0; any time unit (the outputs use the same).  The last
+ *                gap must not be below the one before it (PLOGP_E_RANGE): all predicted times are then >= 0.
  *   latency      HOST, [n_tables]; finite, >= 0.
  *   out          receives the handle; release it with plogp_table_free.
  * The host arrays are copied before the call returns; the caller keeps them.  The call
@@ -172,11 +175,13 @@ const char *plogp_last_cuda_error(void);
  *   d_sizes_bytes  DEVICE, [n_bp] strictly increasing sizes (< 2^53); n_bp <= PLOGP_MAX_BREAKPOINTS
  *   d_gap          DEVICE, [n_bp] finite gaps >= 0
  *   latency        L, finite, >= 0
+ *   P_lo, P_hi     process counts, 2 <= P_lo <= P_hi <= PLOGP_STATIC_MAX_P + 1 (the scan always covers the
+ *                  terms j = 1 .. P_hi - 1, shared by all thread blocks, whatever P_lo is)
  *   d_m_bytes      DEVICE, [n_m] message sizes; n_m <= PLOGP_STATIC_MAX_M; P_hi * m must stay < 2^53
  *   d_time         DEVICE, [P_hi - P_lo + 1][n_m] doubles, m fastest; owned by the caller
  *   stream         cudaStream_t the three kernels are enqueued on; the call does not wait for them
  * The contents of the device arrays cannot be checked on the host and are trusted.  Sizes beyond
- * the stated maxima (n_m, P_hi - P_lo + 1 <= PLOGP_STATIC_MAX_P, n_bp) return PLOGP_E_RANGE; other
+ * the stated maxima (n_m, P_hi - 1 <= PLOGP_STATIC_MAX_P, n_bp) return PLOGP_E_RANGE; other
  * malformed arguments PLOGP_E_INVAL.
  * The first call on each device looks up the array's device address (with that device current);
  * make that first call outside any stream capture.  All calls on a device share the array, which

@@ -36,6 +36,7 @@ int cuda_fail(cudaError_t e, const char *what)
 constexpr uint32_t kSegBits = (1u << 2) | (1u << 5) | (1u << 9);
 constexpr uint64_t kTwo32 = 1ull << 32;
 constexpr double kTwo53 = 9007199254740992.0;
+constexpr int64_t kMaxP = int64_t(1) << 30;  // process counts: 32-bit tiling arithmetic and 1 << ceil(log2 P) stay in range
 constexpr size_t kSweepScratchLimit = size_t(1) << 30;  // per launch batch of tables
 
 int ceil_log2(int64_t P)
@@ -158,6 +159,7 @@ int validate_grid(const plogp_tables *h, const plogp_grid *g, int64_t *n_s_out)
         if (g->P_lo < 2 || g->P_hi < g->P_lo) return PLOGP_E_INVAL;
         P_hi = g->P_hi;
     }
+    if (P_hi > kMaxP) return PLOGP_E_RANGE;
     for (int i = 0; i < g->n_m; ++i) {
         const uint64_t m = g->m[i];
         if (m == 0 || m % g->dtype_bytes) return PLOGP_E_INVAL;
@@ -415,7 +417,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             dp.T = h->T; dp.G = pl.G;
             dp.G.mask &= 0x3FFu;
             dp.n_mgroups = pl.dec_mgroups; dp.n_ptiles = pl.dec_ptiles; dp.mg = pl.dec_mg;
-            dp.table0 = t0; dp.n_tables_launch = nt;
+            dp.table0 = t0; dp.n_tables_launch = nt; dp.out_table0 = out.out_table0;
             dp.d_strategy = out.d_strategy; dp.d_sbytes = out.d_sbytes; dp.d_time = out.d_time;
             dp.vec_out = (pl.G.n_m % 2 == 0) && pl.dec_mg >= 2 && reinterpret_cast<uintptr_t>(out.d_time) % 16 == 0 &&
                          reinterpret_cast<uintptr_t>(out.d_sbytes) % 8 == 0 && reinterpret_cast<uintptr_t>(out.d_strategy) % 2 == 0;
@@ -465,6 +467,9 @@ static int build_tables(int n_tables, int n_bp, int npad, const uint64_t *sizes_
             if (i && sz[i] <= sz[i - 1]) return PLOGP_E_INVAL;
             if (double(sz[i]) >= kTwo53) return PLOGP_E_RANGE;
         }
+        // Above the last size the last interval's line is continued: a falling line would turn g negative for
+        // large arguments, and the kernels compare times through their (sign-free) high words.
+        if (gp[n_bp - 1] < gp[n_bp - 2]) return PLOGP_E_RANGE;
         double *key = tab.data() + size_t(t) * 3 * npad, *g0 = key + npad, *sl = g0 + npad;
         for (int i = 0; i < npad; ++i) {
             if (i <= n_bp - 2) {
@@ -645,23 +650,33 @@ int plogp_select_best_host(plogp_tables *h, const plogp_grid *grid, uint8_t *h_s
         double *s_time = reinterpret_cast<double *>(h->d_stage[slot]);
         uint32_t *s_sb = reinterpret_cast<uint32_t *>(h->d_stage[slot] + align(cells * 8 * batch));
         uint8_t *s_id = h->d_stage[slot] + align(cells * 8 * batch) + align(cells * 4 * batch);
-        if (t0 >= 2 * batch) CK(cudaStreamWaitEvent(st, h->ev_copied[slot], 0));  // the set's previous copy has left
+        if (t0 >= 2 * batch) {  // the set's previous copy has left
+            cudaError_t ew = cudaStreamWaitEvent(st, h->ev_copied[slot], 0);
+            if (ew != cudaSuccess) { rc = cuda_fail(ew, "cudaStreamWaitEvent"); break; }
+        }
         FusedParams out{};
-        // the kernels index outputs by absolute table number
-        out.d_time = s_time - size_t(t0) * cells;
-        out.d_sbytes = s_sb - size_t(t0) * cells;
-        out.d_strategy = s_id - size_t(t0) * cells;
+        out.d_time = s_time;
+        out.d_sbytes = s_sb;
+        out.d_strategy = s_id;
+        out.out_table0 = t0;  // the staging set holds tables t0 .. t0 + nt - 1
         rc = run(h, grid, false, out, st, t0, t0 + nt);
+        // On any failure the loop ends here, and both streams are drained below before the call returns: no
+        // copy into the caller's arrays is left in flight.
+        cudaError_t e = cudaSuccess;
+        if (rc == PLOGP_OK) e = cudaEventRecord(h->ev_done[slot], st);
+        if (rc == PLOGP_OK && e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_stream, h->ev_done[slot], 0);
+        if (rc == PLOGP_OK && e == cudaSuccess)
+            e = cudaMemcpyAsync(h_time + size_t(t0) * cells, s_time, cells * 8 * nt, cudaMemcpyDeviceToHost, h->copy_stream);
+        if (rc == PLOGP_OK && e == cudaSuccess)
+            e = cudaMemcpyAsync(h_s_bytes + size_t(t0) * cells, s_sb, cells * 4 * nt, cudaMemcpyDeviceToHost, h->copy_stream);
+        if (rc == PLOGP_OK && e == cudaSuccess)
+            e = cudaMemcpyAsync(h_strategy + size_t(t0) * cells, s_id, cells * nt, cudaMemcpyDeviceToHost, h->copy_stream);
+        if (rc == PLOGP_OK && e == cudaSuccess) e = cudaEventRecord(h->ev_copied[slot], h->copy_stream);
+        if (rc == PLOGP_OK && e != cudaSuccess) rc = cuda_fail(e, "plogp_select_best_host: copy pipeline");
         if (rc != PLOGP_OK) break;
-        CK(cudaEventRecord(h->ev_done[slot], st));
-        CK(cudaStreamWaitEvent(h->copy_stream, h->ev_done[slot], 0));
-        CK(cudaMemcpyAsync(h_time + size_t(t0) * cells, s_time, cells * 8 * nt, cudaMemcpyDeviceToHost, h->copy_stream));
-        CK(cudaMemcpyAsync(h_s_bytes + size_t(t0) * cells, s_sb, cells * 4 * nt, cudaMemcpyDeviceToHost, h->copy_stream));
-        CK(cudaMemcpyAsync(h_strategy + size_t(t0) * cells, s_id, cells * nt, cudaMemcpyDeviceToHost, h->copy_stream));
-        CK(cudaEventRecord(h->ev_copied[slot], h->copy_stream));
     }
     cudaError_t e1 = cudaStreamSynchronize(h->copy_stream), e2 = cudaStreamSynchronize(st);
-    if (rc != PLOGP_OK) return rc;
+    if (rc != PLOGP_OK) { cudaGetLastError(); return rc; }
     if (e1 != cudaSuccess) return cuda_fail(e1, "cudaStreamSynchronize(copy)");
     if (e2 != cudaSuccess) return cuda_fail(e2, "cudaStreamSynchronize");
     return PLOGP_OK;

@@ -359,7 +359,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
         if (mi < n_mi) {
             const uint32_t m_u0 = p.G.m_list[m0 + mi], m_u1 = p.G.m_list[m0 + mi + 1];
             const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
-            const size_t base = static_cast<size_t>(table) * 2 * plane + static_cast<size_t>(m0 + mi);
+            const size_t base = static_cast<size_t>(table - p.out_table0) * 2 * plane + static_cast<size_t>(m0 + mi);
             const double *st0 = sm.st_time + mi * kStageStride, *st1 = st0 + kStageStride;
             const uint16_t *sc0 = sm.st_code + mi * kCodeStride, *sc1 = sc0 + kCodeStride;
             for (int pr = warp * rows + prow; pr < n_valid; pr += kDecWarps * rows) {
@@ -378,7 +378,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
         if (mi < n_mi) {
             const uint32_t m_u = p.G.m_list[m0 + mi];
             const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
-            const size_t base = static_cast<size_t>(table) * 2 * plane + static_cast<size_t>(m0 + mi);
+            const size_t base = static_cast<size_t>(table - p.out_table0) * 2 * plane + static_cast<size_t>(m0 + mi);
             for (int pr = warp * rows + prow; pr < n_valid; pr += kDecWarps * rows) {
                 const size_t o = base + static_cast<size_t>(tile0 + pr) * p.G.n_m;
                 const uint32_t code = sm.st_code[mi * kCodeStride + pr];

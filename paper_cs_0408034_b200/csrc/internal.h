@@ -53,6 +53,7 @@ struct FusedParams {
     GridDev G;
     int n_mtiles, n_ptiles, passes_per_tile;  // a pass covers kWarps*R process counts
     int table0, n_tables_launch;
+    int out_table0;  // table whose results sit at the start of the output arrays (0 unless the caller passes a window)
     const double *s1_carry;  // [n_tables_launch][n_ptiles][n_m] exclusive tile prefixes, or nullptr
     // segmented minima precomputed by the sweep kernel (nullptr => inline sweep)
     const double *part_time;
@@ -84,6 +85,7 @@ struct DecideParams {
     int mg;  // message sizes per CTA, 1..kDecMG
     int vec_out;  // outputs aligned for two message sizes per store (n_m even, 16 / 8 / 2-byte aligned bases)
     int table0, n_tables_launch;
+    int out_table0;  // table whose results sit at the start of the output arrays
     uint8_t *d_strategy;
     uint32_t *d_sbytes;
     double *d_time;

@@ -415,7 +415,7 @@ __global__ void __launch_bounds__(kThreads) fused_kernel(const FusedParams p)
         for (int r = 0; r < R; ++r) { bt[r] = CUDART_INF; bsz[r] = 0; bid[r] = 255; }
 
         auto out_index = [&](int id_or_coll, int planes, int r) {
-            return (static_cast<size_t>(table) * planes + id_or_coll) * plane +
+            return (static_cast<size_t>(table - p.out_table0) * planes + id_or_coll) * plane +
                    static_cast<size_t>(p0 + r) * p.G.n_m + midx;
         };
         auto consider = [&](int id, const double *val, const uint32_t *sval) {

@@ -9,6 +9,7 @@
 #include "../../include/plogp.h"
 
 #include <cuda_runtime.h>
+#include <cmath>
 #include <mutex>
 
 namespace {
@@ -28,6 +29,9 @@ constexpr int kMaxDevices = 64;
 // address is fetched once per device with cudaGetSymbolAddress and passed to the kernels.
 static __device__ __align__(256) double g_static_scratch[kNaScratchDoubles];
 
+// The scan runs over the terms j = 1 .. P_hi - 1 of the sum, whatever P_lo is: term index e stands for j = e + 1,
+// i.e. for the process count P = e + 2, and rows below P_lo are simply not written.  All CTAs share the work
+// for the terms below P_lo that way, and no thread ever owns more than one term per index.
 struct NaArgs {
     const uint64_t *sizes;
     const double *gap;
@@ -35,7 +39,7 @@ struct NaArgs {
     double *time;
     double *scratch;
     double L;
-    int n_bp, npad, P_lo, n_P, n_m, n_mtiles, n_ptiles;
+    int n_bp, npad, P_lo, n_terms, n_m, n_mtiles, n_ptiles;
 };
 
 // key | gap | slope in shared memory, built from the caller's raw table
@@ -86,27 +90,15 @@ __global__ void __launch_bounds__(kNaThreads) na_chain_kernel(const NaArgs a)
     double carry = (PHASE == 3 && m_ok) ? a.scratch[ptile * a.n_m + midx] : 0.0;
     double acc = 0.0;
     for (int pass = 0; pass < kNaPasses; ++pass) {
-        const int p_cta = ptile * kNaTileP + pass * kNaPassP;
-        if (p_cta >= a.n_P) break;
-        const int p0 = p_cta + warp * kNaR;
+        const int e_cta = ptile * kNaTileP + pass * kNaPassP;
+        if (e_cta >= a.n_terms) break;
+        const int e0 = e_cta + warp * kNaR;
         double pre[kNaR];
         double run = 0.0;
 #pragma unroll
         for (int r = 0; r < kNaR; ++r) {
-            const int pidx = p0 + r;
-            if (pidx < a.n_P) {
-                // term of index pidx: j runs from the previous process count (1 before the first) to P-1
-                const int jhi = a.P_lo + pidx - 1;
-                int j = pidx == 0 ? 1 : jhi;
-                double comp = 0.0, sum = 0.0;
-                for (; j <= jhi; ++j) {
-                    const double y = na_gap(s_tab, a.npad, static_cast<double>(j) * md) - comp;
-                    const double t = sum + y;
-                    comp = (t - sum) - y;
-                    sum = t;
-                }
-                run += sum;
-            }
+            const int e = e0 + r;
+            if (e < a.n_terms) run += na_gap(s_tab, a.npad, static_cast<double>(e + 1) * md);  // g(j m), j = e + 1
             pre[r] = run;
         }
         if (PHASE == 1) {
@@ -124,10 +116,11 @@ __global__ void __launch_bounds__(kNaThreads) na_chain_kernel(const NaArgs a)
             }
 #pragma unroll
             for (int r = 0; r < kNaR; ++r) {
-                const int pidx = p0 + r;
-                if (pidx < a.n_P && m_ok)
-                    a.time[static_cast<size_t>(pidx) * a.n_m + midx] =
-                        fma(static_cast<double>(a.P_lo + pidx - 1), a.L, carry + before + pre[r]);
+                const int e = e0 + r;
+                const int P = e + 2;  // the sum up to j = e + 1 = P - 1 belongs to this process count
+                if (e < a.n_terms && P >= a.P_lo && m_ok)
+                    a.time[static_cast<size_t>(P - a.P_lo) * a.n_m + midx] =
+                        fma(static_cast<double>(P - 1), a.L, carry + before + pre[r]);
             }
             carry += all;
         }
@@ -167,9 +160,9 @@ extern "C" int plogp_scatter_chain_static(int n_bp, const uint64_t *d_sizes_byte
                                           const uint64_t *d_m_bytes, int32_t n_m, double *d_time, void *stream)
 {
     if (!d_sizes_bytes || !d_gap || !d_m_bytes || !d_time) return PLOGP_E_INVAL;
-    if (n_bp < 2 || P_lo < 2 || P_hi < P_lo || n_m < 1 || !(latency >= 0.0)) return PLOGP_E_INVAL;
-    const long long n_P = static_cast<long long>(P_hi) - P_lo + 1;
-    if (n_bp > PLOGP_MAX_BREAKPOINTS || n_m > PLOGP_STATIC_MAX_M || n_P > PLOGP_STATIC_MAX_P) return PLOGP_E_RANGE;
+    if (n_bp < 2 || P_lo < 2 || P_hi < P_lo || n_m < 1 || !std::isfinite(latency) || latency < 0.0) return PLOGP_E_INVAL;
+    const long long n_terms = static_cast<long long>(P_hi) - 1;  // j = 1 .. P_hi - 1
+    if (n_bp > PLOGP_MAX_BREAKPOINTS || n_m > PLOGP_STATIC_MAX_M || n_terms > PLOGP_STATIC_MAX_P) return PLOGP_E_RANGE;
 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return PLOGP_E_CUDA;
@@ -191,11 +184,11 @@ extern "C" int plogp_scatter_chain_static(int n_bp, const uint64_t *d_sizes_byte
 
     NaArgs a{};
     a.sizes = d_sizes_bytes; a.gap = d_gap; a.m = d_m_bytes; a.time = d_time; a.scratch = scratch;
-    a.L = latency; a.n_bp = n_bp; a.P_lo = P_lo; a.n_P = static_cast<int>(n_P); a.n_m = n_m;
+    a.L = latency; a.n_bp = n_bp; a.P_lo = P_lo; a.n_terms = static_cast<int>(n_terms); a.n_m = n_m;
     a.npad = 2;
     while (a.npad < n_bp - 1) a.npad <<= 1;
     a.n_mtiles = (n_m + 31) / 32;
-    a.n_ptiles = (a.n_P + kNaTileP - 1) / kNaTileP;
+    a.n_ptiles = (a.n_terms + kNaTileP - 1) / kNaTileP;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t smem = (3 * static_cast<size_t>(a.npad) + 2 * kNaWarps * 32) * sizeof(double);  // <= 28 KiB

@@ -71,6 +71,8 @@ def test_table_validation_runs_on_the_host_before_any_device_call():
     assert status([4, 8, 16], [[1.0, 2.0, 3.0]], [-1.0]) == plogp.E_INVAL
     assert status([4], [[1.0]], [1.0]) == plogp.E_INVAL
     assert status([4, 8, 1 << 60], [[1.0, 2.0, 3.0]], [1.0]) == plogp.E_RANGE
+    assert status([4, 8, 16], [[1.0, 3.0, 2.0]], [1.0]) == plogp.E_RANGE   # falling last interval: g would turn negative above the table
+    assert status([4, 8, 16], [[1.0, 3.0, 2.0]], [float("inf")]) == plogp.E_INVAL
     assert status([[4, 8, 16], [4, 8, 8]], [[1.0, 2.0, 3.0], [1.0, 2.0, 3.0]], [1.0, 1.0], shared=0) == plogp.E_INVAL
     h = ctypes.c_void_p()
     assert plogp.lib.plogp_table_load(1, 3, None, 1, None, None, ctypes.byref(h)) == plogp.E_INVAL

@@ -41,6 +41,7 @@ def test_bad_tables(plogp):
     assert load_status(plogp, [4, 8, 16], ok[1], [np.inf]) == plogp.E_INVAL
     assert load_status(plogp, [4], [[1.0]], [1.0]) == plogp.E_INVAL             # fewer than two sizes
     assert load_status(plogp, [4, 8, 1 << 60], ok[1], ok[2]) == plogp.E_RANGE
+    assert load_status(plogp, [4, 8, 16], [[1.0, 3.0, 2.5]], [1.0]) == plogp.E_RANGE   # falling last interval
     n = 1025
     assert load_status(plogp, np.arange(1, n + 1) * 4, [np.arange(n, dtype=np.float64)], [1.0]) == plogp.E_RANGE
     h = C.c_void_p()
@@ -64,6 +65,8 @@ def test_bad_grids_and_null_outputs(plogp):
         assert status() == plogp.OK
         assert status(P_lo=1) == plogp.E_INVAL
         assert status(P_lo=6, P_hi=5) == plogp.E_INVAL
+        assert status(P_lo=(1 << 30) - 2, P_hi=(1 << 30) + 1, m=[4], s=[4]) == plogp.E_RANGE   # process counts above 2^30
+        assert status(P=[2, (1 << 30) + 1], m=[4], s=[4]) == plogp.E_RANGE
         assert status(P=[2, 2, 3]) == plogp.E_INVAL
         assert status(P=[3, 1]) == plogp.E_INVAL
         assert status(m=[16, 8]) == plogp.E_INVAL
