@@ -205,7 +205,7 @@ int plogp_scatter_chain_static(int n_bp, const uint64_t *d_sizes_bytes, const do
  */
 enum {
     PLOGP_KERNEL_SWEEP = 0,        /* segment sweep over long candidate lists */
-    PLOGP_KERNEL_CHAIN_PREFIX = 1, /* Scatter Chain tile sums + their scan (two launches, timed together) */
+    PLOGP_KERNEL_CHAIN_PREFIX = 1, /* Scatter Chain sums per tile of process counts (when P is split over thread blocks) */
     PLOGP_KERNEL_FUSED = 2,        /* all strategies, lanes <-> m (predictions, long lists' final pass) */
     PLOGP_KERNEL_DECIDE = 3,       /* Broadcast decision, lanes <-> P (short candidate lists) */
     PLOGP_KERNEL_SCATTER = 4,      /* Scatter decision */

@@ -56,6 +56,9 @@ struct Plan {
     bool inline_sweep = true;
     // fused kernel tiling
     int n_mtiles = 0, n_ptiles = 1, passes_per_tile = 1;
+    // Scatter decision kernel: its own split of P (one CTA run covers a short P range in a few microseconds,
+    // and an unsplit range needs no tile sums, i.e. one launch less)
+    int sc_ptiles = 1, sc_passes_per_tile = 1;
     // decision kernel tiling (short candidate lists)
     int dec_mgroups = 0, dec_ptiles = 1, dec_mg = kDecMG;
     size_t carry_bytes_per_table = 0;
@@ -260,6 +263,8 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     n_ptiles = std::min(n_ptiles, 256);
     pl.passes_per_tile = (total_passes + n_ptiles - 1) / n_ptiles;
     pl.n_ptiles = (total_passes + pl.passes_per_tile - 1) / pl.passes_per_tile;
+    if (n_P <= 512) { pl.sc_ptiles = 1; pl.sc_passes_per_tile = total_passes; }
+    else { pl.sc_ptiles = pl.n_ptiles; pl.sc_passes_per_tile = pl.passes_per_tile; }
 
     pl.dec_ptiles = (n_P + kDecTileP - 1) / kDecTileP;
     // 16 message sizes per CTA give the widest output rows; small grids trade that for more CTAs
@@ -336,7 +341,7 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     const bool s1_on = (g->strategy_mask >> 11) & 1u;
     size_t per_table = 0;
     if (!pl.inline_sweep) per_table += size_t(pl.n_seg) * pl.n_pairs * n_P * (sizeof(double) + sizeof(uint32_t)) + 512;
-    if (s1_on && pl.n_ptiles > 1) pl.carry_bytes_per_table = size_t(pl.n_ptiles) * n_m * sizeof(double);
+    if (s1_on && pl.n_ptiles > 1) pl.carry_bytes_per_table = size_t(pl.n_ptiles) * (kWarps + 1) * n_m * sizeof(double);
     per_table += pl.carry_bytes_per_table;
     pl.tables_per_batch = h->T.n_tables;
     if (!pl.inline_sweep && per_table * h->T.n_tables > kSweepScratchLimit)
@@ -371,8 +376,10 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
     // Short candidate lists with segmented strategies: the lane<->P decision kernel; everything else
     // (predictions, long lists reduced by the sweep kernel, Scatter-only grids) goes through fused_kernel.
     const bool use_decide = !predict && pl.inline_sweep && pl.n_seg > 0;
-    const int n_ptiles = pl.n_ptiles;
-    const int passes_per_tile = pl.passes_per_tile;
+    // the kernel that follows the (optional) Broadcast decision kernel: Scatter strategies only => scatter_kernel
+    const bool use_scatter = !predict && ((use_decide ? pl.G.mask & 0x1C00u : pl.G.mask) & 0x3FFu) == 0;
+    const int n_ptiles = use_scatter ? pl.sc_ptiles : pl.n_ptiles;
+    const int passes_per_tile = use_scatter ? pl.sc_passes_per_tile : pl.passes_per_tile;
     const bool need_carry = s1 && n_ptiles > 1;
 
     if (t_end < 0) t_end = h->T.n_tables;
@@ -408,7 +415,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             s.n_mtiles = pl.n_mtiles; s.n_ptiles = n_ptiles; s.passes_per_tile = passes_per_tile;
             s.table0 = t0; s.n_tables_launch = nt; s.tile_sum = tile_sum;
             { LaunchTimer lt(h, PLOGP_KERNEL_CHAIN_PREFIX, st); CK(launch_s1_tiles(s, st)); }
-            g_launches += 2;
+            g_launches += 1;
         }
         GridDev Gf = pl.G;
         if (use_decide) {
@@ -429,15 +436,15 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
         }
         FusedParams fp = out;
         fp.T = h->T; fp.G = Gf;
-        fp.n_mtiles = pl.n_mtiles; fp.n_ptiles = pl.n_ptiles; fp.passes_per_tile = pl.passes_per_tile;
+        fp.n_mtiles = pl.n_mtiles; fp.n_ptiles = n_ptiles; fp.passes_per_tile = passes_per_tile;
         fp.table0 = t0; fp.n_tables_launch = nt;
-        fp.s1_carry = tile_sum;
+        fp.s1_sums = tile_sum;
         // part_time doubles as the "segmented minima come from the sweep kernel" switch
         fp.part_time = pl.inline_sweep ? nullptr : part_time;
         fp.part_idx = part_idx;
         fp.pair_base = pl.inline_sweep ? nullptr : reinterpret_cast<const int32_t *>(h->d_grid + pl.off_pair_base);
         fp.n_pairs = pl.n_pairs; fp.n_seg = pl.n_seg;
-        if (!predict && (Gf.mask & 0x3FFu) == 0) { LaunchTimer lt(h, PLOGP_KERNEL_SCATTER, st); CK(launch_scatter(fp, st)); }
+        if (use_scatter) { LaunchTimer lt(h, PLOGP_KERNEL_SCATTER, st); CK(launch_scatter(fp, st)); }
         else { LaunchTimer lt(h, PLOGP_KERNEL_FUSED, st); CK(launch_fused(fp, predict, st)); }
         g_launches += 1;
     }

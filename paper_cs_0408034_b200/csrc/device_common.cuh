@@ -126,4 +126,24 @@ __device__ __forceinline__ double s1_term(const double *s_tab, int npad, const G
     return sum;
 }
 
+// Scatter Chain sum in front of a warp's run when the P range is split over CTAs: the totals of the tiles
+// in front of this one (added up by the CTA's warps in a fixed order: warp w takes tiles w, w + 8, ...) plus
+// the shares of the lower warps of this tile.  sums is laid out [table][tile][9][m] (8 warp shares, then the
+// tile's total); s_buf holds kWarps * 32 doubles.  Called by all threads of the CTA (one barrier inside).
+__device__ __forceinline__ double chain_prefix(const double *sums, int trel, int n_ptiles, int ptile, int warp, int lane,
+                                               int n_m, int midx_c, double *s_buf)
+{
+    const double *tab0 = sums + static_cast<size_t>(trel) * n_ptiles * (kWarps + 1) * n_m + midx_c;
+    double part = 0.0;
+    for (int t = warp; t < ptile; t += kWarps) part += tab0[(static_cast<size_t>(t) * (kWarps + 1) + kWarps) * n_m];
+    s_buf[warp * 32 + lane] = part;
+    __syncthreads();
+    double run = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) run += s_buf[w * 32 + lane];
+    const double *mine = tab0 + static_cast<size_t>(ptile) * (kWarps + 1) * n_m;
+    for (int w = 0; w < warp; ++w) run += mine[static_cast<size_t>(w) * n_m];
+    return run;
+}
+
 }  // namespace plogp

@@ -54,7 +54,7 @@ struct FusedParams {
     int n_mtiles, n_ptiles, passes_per_tile;  // a pass covers kWarps*R process counts
     int table0, n_tables_launch;
     int out_table0;  // table whose results sit at the start of the output arrays (0 unless the caller passes a window)
-    const double *s1_carry;  // [n_tables_launch][n_ptiles][n_m] exclusive tile prefixes, or nullptr
+    const double *s1_sums;  // [n_tables_launch][n_ptiles][9][n_m] Scatter Chain sums per warp run and per tile, or nullptr
     // segmented minima precomputed by the sweep kernel (nullptr => inline sweep)
     const double *part_time;
     const uint32_t *part_idx;
@@ -74,7 +74,7 @@ struct S1Params {
     GridDev G;
     int n_mtiles, n_ptiles, passes_per_tile;
     int table0, n_tables_launch;
-    double *tile_sum;  // [n_tables_launch][n_ptiles][n_m]
+    double *tile_sum;  // [n_tables_launch][n_ptiles][9][n_m]: the 8 warps' shares, then the tile's total
 };
 
 // Decision kernel for short candidate lists (lanes <-> P): see decide.cu

@@ -12,7 +12,8 @@
 //                  candidate lists inline or reduces the sweep kernel's partial minima, keeps the
 //                  Scatter Chain sum running along each warp's contiguous run of P, and writes either
 //                  the predicted planes or the decision table.  The general path.
-//   s1_tile_*      tile sums and their scan for the Scatter Chain sum when P is split over CTAs.
+//   s1_tile_sum    per-tile and per-warp-run sums for the Scatter Chain sum when P is split over CTAs
+//                  (reduce-then-scan: the consumers add up the sums of the tiles in front of theirs).
 // The decision table of short candidate lists has faster, specialised kernels in decide.cu
 // (Broadcast half) and scatter.cu (Scatter half).
 #include "device_common.cuh"
@@ -223,47 +224,19 @@ __global__ void __launch_bounds__(kThreads) s1_tile_sum_kernel(const S1Params p)
     const int p_warp = ptile * (kWarps * run_len) + warp * run_len;
     for (int e = 0; e < run_len; ++e)
         if (p_warp + e < p.G.n_P) acc += s1_term(s_tab, p.T.npad, p.G, p_warp + e, md, walk);
+    // Per tile and message size: the shares of the 8 warps (each the sum over its run of process counts) and
+    // their total, laid out as [tile][9][m]; the kernels that follow turn them into the sum in front of a run.
     s_red[warp * 32 + lane] = acc;
     __syncthreads();
-    if (warp == 0 && midx < p.G.n_m) {
-        double t = 0.0;
+    if (midx < p.G.n_m) {
+        double *row = p.tile_sum + (static_cast<size_t>(trel) * p.n_ptiles + ptile) * (kWarps + 1) * p.G.n_m + midx;
+        row[static_cast<size_t>(warp) * p.G.n_m] = acc;
+        if (warp == 0) {
+            double t = 0.0;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) t += s_red[w * 32 + lane];
-        p.tile_sum[(static_cast<size_t>(trel) * p.n_ptiles + ptile) * p.G.n_m + midx] = t;
-    }
-}
-
-// Exclusive scan of the tile sums along the tile index, in place: one warp per (table, m), each lane a
-// contiguous block of at most kScanPerLane tiles (n_ptiles <= 32 * kScanPerLane = 256).
-constexpr int kScanPerLane = 8;
-__global__ void s1_tile_scan_kernel(double *tile_sum, int n_tables, int n_ptiles, int n_m)
-{
-    const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    if (i >= n_tables * n_m) return;  // whole warps leave together
-    const int trel = i / n_m, midx = i - trel * n_m;
-    const int per = (n_ptiles + 31) / 32;
-    double *base = tile_sum + static_cast<size_t>(trel) * n_ptiles * n_m + midx;
-    double v[kScanPerLane];
-    double mine = 0.0;
-#pragma unroll
-    for (int k = 0; k < kScanPerLane; ++k) {
-        const int pt = lane * per + k;
-        v[k] = (k < per && pt < n_ptiles) ? base[static_cast<size_t>(pt) * n_m] : 0.0;
-        mine += v[k];
-    }
-    double incl = mine;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const double y = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += y;
-    }
-    double run = __shfl_up_sync(0xffffffffu, incl, 1);  // sum of the lower lanes' blocks
-    if (lane == 0) run = 0.0;
-#pragma unroll
-    for (int k = 0; k < kScanPerLane; ++k) {
-        const int pt = lane * per + k;
-        if (k < per && pt < n_ptiles) base[static_cast<size_t>(pt) * n_m] = run;
-        run += v[k];
+            for (int w = 0; w < kWarps; ++w) t += s_red[w * 32 + lane];
+            row[static_cast<size_t>(kWarps) * p.G.n_m] = t;
+        }
     }
 }
 
@@ -367,18 +340,22 @@ __global__ void __launch_bounds__(kThreads) fused_kernel(const FusedParams p)
     const int run_len = p.passes_per_tile * R;
     const int p_warp = ptile * (kWarps * run_len) + warp * run_len;
 
-    // Scatter Chain: prefix of g(j m) in front of this thread's run = tile carry + the runs of the lower warps
+    // Scatter Chain: prefix of g(j m) in front of this thread's run = the tiles in front (sums from
+    // s1_tile_sum_kernel when the P range is split over CTAs) + the runs of the lower warps
     double s1_run = 0.0;
     GapWalk s1_walk;  // table interval of this thread's last Scatter Chain argument
     if ((mask >> 11) & 1u) {
-        double mine = 0.0;
-        for (int e = 0; e < run_len; ++e)
-            if (p_warp + e < p.G.n_P) mine += s1_term(sm.tab, npad, p.G, p_warp + e, md, s1_walk);
-        sm.tot[warp * 32 + lane] = mine;
-        __syncthreads();
-        if (p.s1_carry) s1_run = p.s1_carry[(static_cast<size_t>(trel) * p.n_ptiles + ptile) * p.G.n_m + midx_c];
-        for (int w = 0; w < warp; ++w) s1_run += sm.tot[w * 32 + lane];
-        s1_walk.i = -1;
+        if (p.s1_sums) {
+            s1_run = chain_prefix(p.s1_sums, trel, p.n_ptiles, ptile, warp, lane, p.G.n_m, midx_c, sm.tot);
+        } else {
+            double mine = 0.0;
+            for (int e = 0; e < run_len; ++e)
+                if (p_warp + e < p.G.n_P) mine += s1_term(sm.tab, npad, p.G, p_warp + e, md, s1_walk);
+            sm.tot[warp * 32 + lane] = mine;
+            __syncthreads();
+            for (int w = 0; w < warp; ++w) s1_run += sm.tot[w * 32 + lane];
+            s1_walk.i = -1;
+        }
     }
 
     const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
@@ -661,10 +638,6 @@ cudaError_t launch_s1_tiles(const S1Params &p, cudaStream_t st)
     const long long blocks = static_cast<long long>(p.n_mtiles) * p.n_ptiles * p.n_tables_launch;
     if (blocks <= 0 || blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     s1_tile_sum_kernel<<<static_cast<unsigned>(blocks), kThreads, smem, st>>>(p);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    const int n = p.n_tables_launch * p.G.n_m;
-    if (p.n_ptiles > 32 * kScanPerLane) return cudaErrorInvalidConfiguration;  // the host plan caps the tile count at 256
-    s1_tile_scan_kernel<<<(n + 3) / 4, 128, 0, st>>>(p.tile_sum, p.n_tables_launch, p.n_ptiles, p.G.n_m);
     return cudaGetLastError();
 }
 

@@ -6,8 +6,8 @@
 // the Chain model's sum over j = 1..P-1 of g(j m) into a running sum along the thread: the argument
 // j m grows by m per step, the table interval is kept in registers and only reloaded when the
 // argument crosses a breakpoint.  The sum in front of a warp's run comes from the runs of the lower
-// warps (one pass over the run without stores, one barrier) plus the tile prefix computed by
-// s1_tile_sum_kernel / s1_tile_scan_kernel when the P range is split over several CTAs.
+// warps (one pass over the run without stores, one barrier) or, when the P range is split over
+// several CTAs, from the per-run and per-tile sums that s1_tile_sum_kernel has written (reduce-then-scan).
 #include "device_common.cuh"
 
 namespace plogp {
@@ -125,28 +125,31 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
     const double x_first = static_cast<double>((e0 == 0 || !CONTIG) ? (e0 == 0 ? 1 : P_at(p.G, e0 - 1)) : P0 - 1) * md;
 
     double run = 0.0;
-    if (on11) {  // first pass over the run, no stores: this warp's share of the sum
-        double mine = 0.0;
-        if (e0 < e1) {
-            LineWalk w;
-            w.start(s_tab, npad, x_first);
-            if (CONTIG) {
-                if (e0 == 0) mine = below_first(w);
-                double x = static_cast<double>(P0 - 1) * md;
-                for (int e = e0; e < e1; ++e) {
-                    mine += w.at(s_tab, npad, x);
-                    x += md;  // exact: j m < 2^53
+    if (on11 && p.s1_sums) {
+        // P range split over CTAs: the sums of the tiles and warp runs in front come from s1_tile_sum_kernel
+        run = chain_prefix(p.s1_sums, trel, p.n_ptiles, ptile, warp, lane, p.G.n_m, midx_c, s_tot);  // one barrier inside
+    } else {
+        if (on11) {  // first pass over the run, no stores: this warp's share of the sum
+            double mine = 0.0;
+            if (e0 < e1) {
+                LineWalk w;
+                w.start(s_tab, npad, x_first);
+                if (CONTIG) {
+                    if (e0 == 0) mine = below_first(w);
+                    double x = static_cast<double>(P0 - 1) * md;
+                    for (int e = e0; e < e1; ++e) {
+                        mine += w.at(s_tab, npad, x);
+                        x += md;  // exact: j m < 2^53
+                    }
+                } else {
+                    for (int e = e0; e < e1; ++e) mine += listed_step(e, P_at(p.G, e), w);
                 }
-            } else {
-                for (int e = e0; e < e1; ++e) mine += listed_step(e, P_at(p.G, e), w);
             }
+            s_tot[warp * 32 + lane] = mine;
         }
-        s_tot[warp * 32 + lane] = mine;
-    }
-    __syncthreads();  // also publishes s_cum
-    if (on11) {
-        if (p.s1_carry) run = p.s1_carry[(static_cast<size_t>(trel) * p.n_ptiles + ptile) * p.G.n_m + midx_c];
-        for (int w = 0; w < warp; ++w) run += s_tot[w * 32 + lane];
+        __syncthreads();  // also publishes s_cum
+        if (on11)
+            for (int w = 0; w < warp; ++w) run += s_tot[w * 32 + lane];
     }
     if (e0 >= e1 || !m_ok) return;  // no barriers below
 
