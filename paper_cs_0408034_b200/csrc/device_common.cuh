@@ -107,23 +107,52 @@ struct GapWalk {
     }
 };
 
+// Sum of g(j m) for j = jlo .. jhi (jlo <= jhi) in closed form: inside one table interval g is a line, so the
+// terms whose arguments fall into it are an arithmetic series, n gap_i + slope_i (m (jlo' + jhi') n / 2 - n key_i);
+// the loop runs over the table intervals that the arguments cross (at most n_bp), not over j.  Below the first
+// size g is constant (its first value), above the last size the last interval's line goes on.  This is what
+// keeps a gap in a process-count list, or a first process count far above 2, from turning into a long loop.
+__device__ __forceinline__ double chain_range_sum(const double *s_tab, int npad, double md, long long jlo, long long jhi)
+{
+    double sum = 0.0;
+    long long j = jlo;
+    int i = -1;  // -1: below the table
+    if (static_cast<double>(j) * md >= s_tab[0]) i = interval_of(s_tab, npad, static_cast<double>(j) * md);
+    while (j <= jhi) {
+        const double next = s_tab[i + 1];  // first argument that belongs to the next interval (+inf after the last)
+        long long jend = jhi;
+        if (next <= static_cast<double>(jhi) * md) {
+            // largest j with j m < next (m, next and the products are integers below 2^53: exact)
+            long long q = static_cast<long long>(next / md);
+            while (static_cast<double>(q) * md >= next) --q;
+            while (static_cast<double>(q + 1) * md < next) ++q;
+            jend = q;
+        }
+        if (jend >= j) {
+            const double n = static_cast<double>(jend - j + 1);
+            if (i < 0) {
+                sum += n * s_tab[npad];
+            } else {
+                const double mean = 0.5 * (static_cast<double>(j + jend) * md) - s_tab[i];  // mean argument minus the key
+                sum += n * fma(mean, s_tab[2 * npad + i], s_tab[npad + i]);
+            }
+            j = jend + 1;
+        }
+        ++i;
+    }
+    return sum;
+}
+
 // One term of the Scatter Chain sum for the process count at index pidx: the gaps g(j m) for j
 // from the previous listed process count (1 before the first) up to P-1.  For a contiguous
-// range of P this is the single gap g((P-1) m); longer runs are added with compensation.
+// range of P this is the single gap g((P-1) m); longer runs are summed interval by interval.
 // The walk state must only see non-decreasing arguments.
 __device__ __forceinline__ double s1_term(const double *s_tab, int npad, const GridDev &G, int pidx, double md, GapWalk &w)
 {
     const int jhi = P_at(G, pidx) - 1;
     const int jlo = pidx == 0 ? 1 : P_at(G, pidx - 1);
     if (jlo == jhi) return w.at(s_tab, npad, static_cast<double>(jlo) * md);
-    double sum = 0.0, comp = 0.0;
-    for (int j = jlo; j <= jhi; ++j) {
-        const double y = w.at(s_tab, npad, static_cast<double>(j) * md) - comp;
-        const double t = sum + y;
-        comp = (t - sum) - y;
-        sum = t;
-    }
-    return sum;
+    return chain_range_sum(s_tab, npad, md, jlo, jhi);
 }
 
 // Scatter Chain sum in front of a warp's run when the P range is split over CTAs: the totals of the tiles

@@ -100,26 +100,13 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
     // Chain sum.  Contiguous process counts: the step for index e is the single gap g((P-1) m), and the
     // argument grows by m per step; only the very first index of the grid also owns the gaps below it
     // (j = 1 .. P_lo - 2).  Listed process counts: the step owns all j from the previous count to P-1.
-    auto below_first = [&](LineWalk &w) {  // CONTIG, e0 == 0: sum of g(j m), j = 1 .. P_lo - 2
-        double sum = 0.0, comp = 0.0;
-        for (int j = 1; j <= p.G.P_lo - 2; ++j) {
-            const double y = w.at(s_tab, npad, static_cast<double>(j) * md) - comp;
-            const double t = sum + y;
-            comp = (t - sum) - y;
-            sum = t;
-        }
-        return sum;
+    auto below_first = [&]() {  // CONTIG, e0 == 0: sum of g(j m), j = 1 .. P_lo - 2 (closed form per table interval)
+        return p.G.P_lo > 2 ? chain_range_sum(s_tab, npad, md, 1, p.G.P_lo - 2) : 0.0;
     };
-    auto listed_step = [&](int e, int P, LineWalk &w) {  // !CONTIG
+    auto listed_step = [&](int e, int P, LineWalk &w) {  // !CONTIG: all j from the previous listed count to P - 1
         const int jlo = e == 0 ? 1 : P_at(p.G, e - 1);
-        double sum = 0.0, comp = 0.0;
-        for (int j = jlo; j <= P - 1; ++j) {
-            const double y = w.at(s_tab, npad, static_cast<double>(j) * md) - comp;
-            const double t = sum + y;
-            comp = (t - sum) - y;
-            sum = t;
-        }
-        return sum;
+        if (jlo == P - 1) return w.at(s_tab, npad, static_cast<double>(jlo) * md);
+        return chain_range_sum(s_tab, npad, md, jlo, P - 1);
     };
     const int P0 = e0 < p.G.n_P ? P_at(p.G, e0) : 2;
     const double x_first = static_cast<double>((e0 == 0 || !CONTIG) ? (e0 == 0 ? 1 : P_at(p.G, e0 - 1)) : P0 - 1) * md;
@@ -135,7 +122,7 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
                 LineWalk w;
                 w.start(s_tab, npad, x_first);
                 if (CONTIG) {
-                    if (e0 == 0) mine = below_first(w);
+                    if (e0 == 0) mine = below_first();
                     double x = static_cast<double>(P0 - 1) * md;
                     for (int e = e0; e < e1; ++e) {
                         mine += w.at(s_tab, npad, x);
@@ -156,7 +143,7 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
     LineWalk w;
     if (on11) {
         w.start(s_tab, npad, x_first);
-        if (CONTIG && e0 == 0) run += below_first(w);
+        if (CONTIG && e0 == 0) run += below_first();
     }
     double x = static_cast<double>(P0 - 1) * md;
 

@@ -314,3 +314,16 @@ def test_predict_at_the_batched_launch_shape(plogp):
         assert bool(torch.isfinite(pred.time).all())
     del pred
     torch.cuda.empty_cache()
+
+
+def test_scatter_chain_with_a_far_first_process_count_and_wide_gaps(plogp):
+    """Scatter Chain terms that span thousands of j (a contiguous range that starts far above 2, a
+    process-count list with wide gaps): the library sums them per table interval in closed form, the oracle
+    term by term."""
+    from dataclasses import replace
+    base = wl.config5(P_hi=300, n_m=37)
+    run_both(plogp, replace(base, P_lo=100000, P_hi=100300))
+    P = np.array([2, 3, 5000, 5001, 70000, 70001, 262144, 1000000], dtype=np.int32)
+    run_both(plogp, replace(base, P_lo=2, P_hi=int(P[-1]), P_list=P))
+    # the same through the general kernel (Broadcast strategies enabled as well)
+    run_both(plogp, replace(wl.config2(P_hi=40, n_m=20, n_s=9), P_lo=3000, P_hi=3040))
