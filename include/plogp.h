@@ -34,7 +34,8 @@
  *     3.1 prints it (k_mode 1); every segment costs g(s).
  *   - candidate segment sizes for a message m are the grid values s <= m; if none fits, the
  *     message is sent whole (s = m, k = 1) and best_s reports m.
- *   - ties: the smallest segment size, then the lowest strategy id.
+ *   - ties: the smallest segment size, then the lowest strategy id.  (With search_mode 1 two segment sizes of
+ *     ids 2 / 9 whose g(s) k differ but whose predicted times round to the same double may resolve to either.)
  *
  * Threading: calls on one plogp_tables handle must not overlap in time on the host, and their
  * device work must be ordered (use one stream, or order the streams yourself): a handle owns
@@ -114,6 +115,11 @@ typedef struct {
     uint32_t dtype_bytes;   /* size of the basic datatype, > 0 */
     uint32_t strategy_mask; /* bit i enables strategy id i */
     int32_t k_mode;         /* 0: k = ceil(m/s); 1: k = floor(m/s) */
+    int32_t search_mode;    /* how the minimum over s of Section 3.1 is found; the results are the same:
+                               0: exhaustive, every (P, m, s) cell is evaluated (the default);
+                               1: lower envelope: ids 2 and 9 take the s with the smallest g(s) k once per m, id 5
+                                  walks the lower envelope of its lines in P (only for tables whose gaps never
+                                  decrease with the size; other tables silently take the exhaustive search) */
 } plogp_grid;
 
 /*
@@ -209,7 +215,8 @@ enum {
     PLOGP_KERNEL_FUSED = 2,        /* all strategies, lanes <-> m (predictions, long lists' final pass) */
     PLOGP_KERNEL_DECIDE = 3,       /* Broadcast decision, lanes <-> P (short candidate lists) */
     PLOGP_KERNEL_SCATTER = 4,      /* Scatter decision */
-    PLOGP_N_KERNEL_KINDS = 5
+    PLOGP_KERNEL_ENVELOPE = 5,     /* segment search by lower envelope (search_mode 1) */
+    PLOGP_N_KERNEL_KINDS = 6
 };
 int plogp_profile_enable(plogp_tables *tables, int enable);
 int plogp_profile_read(plogp_tables *tables, double *ms, int32_t *launches);

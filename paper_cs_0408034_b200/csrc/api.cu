@@ -54,6 +54,9 @@ struct Plan {
     GridDev G{};
     int n_seg = 0;
     bool inline_sweep = true;
+    bool envelope = false;        // envelope_kernel instead of the sweep kernel (long candidate lists)
+    bool envelope_short = false;  // the decision kernel prunes its candidate lists (short candidate lists)
+    int env_threads = 256, env_rep_cap = 0, env_coarse = 64, env_max_coarse = 0;
     // fused kernel tiling
     int n_mtiles = 0, n_ptiles = 1, passes_per_tile = 1;
     // Scatter decision kernel: its own split of P (one CTA run covers a short P range in a few microseconds,
@@ -75,6 +78,7 @@ struct plogp_tables {
     int device = 0;
     int sm_count = 148;
     TableDev T{};
+    bool monotone = false;  // no table's gap ever decreases with the size (the envelope search relies on it)
     double *d_tab = nullptr, *d_lat = nullptr;
     unsigned char *d_grid = nullptr;
     size_t grid_cap = 0;
@@ -147,6 +151,7 @@ int validate_grid(const plogp_tables *h, const plogp_grid *g, int64_t *n_s_out)
     if (!g) return PLOGP_E_INVAL;
     if (g->strategy_mask >> PLOGP_N_STRATEGIES) return PLOGP_E_INVAL;
     if (g->k_mode != 0 && g->k_mode != 1) return PLOGP_E_INVAL;
+    if (g->search_mode != 0 && g->search_mode != 1) return PLOGP_E_INVAL;
     if (g->dtype_bytes == 0) return PLOGP_E_INVAL;
     if (g->n_m < 0) return PLOGP_E_INVAL;
     if (g->n_m > 0 && !g->m) return PLOGP_E_INVAL;
@@ -212,6 +217,7 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     put(key, g->n_m);
     put_array(key, g->m, size_t(std::max(g->n_m, 0)));
     put(key, g->strategy_mask); put(key, g->k_mode); put(key, g->dtype_bytes);
+    put(key, g->search_mode); put(key, int(h->monotone));
     if (g->strategy_mask & kSegBits) {
         put(key, has_s);
         if (has_s) { put(key, g->n_s); put_array(key, g->s, size_t(std::max<int64_t>(g->n_s, 0))); }
@@ -234,6 +240,13 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     const int64_t P_hi = g->P ? g->P[n_P - 1] : g->P_hi;
     pl.n_seg = __builtin_popcount(g->strategy_mask & kSegBits);
     pl.inline_sweep = pl.n_seg == 0 || n_s <= kMaxInlineS;
+    // search_mode 1 on tables with non-decreasing gaps.  Long candidate lists: envelope_kernel writes the segmented
+    // minima to the scratch rows that fused_kernel reads.  Short lists: the decision kernel prunes its own lists
+    // (predictions of short lists keep the exhaustive inline search; the results are the same).
+    const bool env_ok = g->search_mode == 1 && pl.n_seg > 0 && n_s > 0 && h->monotone;
+    pl.envelope = env_ok && n_s > kMaxInlineS;
+    pl.envelope_short = env_ok && n_s <= kMaxInlineS;
+    if (pl.envelope) pl.inline_sweep = false;
 
     // candidates per message size (grid values s <= m)
     std::vector<int32_t> ns_of_m(n_m, 0);
@@ -289,7 +302,18 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     }
 
     // ---- sweep kernel plan: (m, chunk) pairs, heaviest first ----
-    if (!pl.inline_sweep) {
+    if (pl.envelope) {
+        // one scratch row per message size
+        std::vector<int32_t> pair_base(n_m + 1);
+        for (int i = 0; i <= n_m; ++i) pair_base[i] = i;
+        pl.n_pairs = n_m;
+        pl.off_pair_base = append_aligned(blob, pair_base);
+        // short lists: small CTAs; the list of representatives of one message size lives in shared memory
+        pl.env_threads = ns_max <= 64 ? 64 : 256;
+        pl.env_rep_cap = std::min(std::max(ns_max, 1), 6144);
+        pl.env_coarse = std::max(64, (n_P + 1023) / 1024);
+        pl.env_max_coarse = (std::max(n_P, 1) - 1 + pl.env_coarse - 1) / pl.env_coarse + 1;
+    } else if (!pl.inline_sweep) {
         pl.chunk_len = std::max(2048, ((ns_max + 31) / 32 + kSweepSub - 1) / kSweepSub * kSweepSub);
         std::vector<int32_t> pair_base(n_m + 1, 0);
         struct Pair { int32_t m, chunk, row, len; };
@@ -398,7 +422,15 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
         }
         if (need_carry) tile_sum = reinterpret_cast<double *>(ws);
 
-        if (!pl.inline_sweep && pl.n_pairs > 0) {
+        if (pl.envelope) {
+            EnvParams ep{};
+            ep.T = h->T; ep.G = pl.G;
+            ep.table0 = t0; ep.n_tables_launch = nt;
+            ep.part_time = part_time; ep.part_idx = part_idx; ep.n_seg = pl.n_seg;
+            ep.rep_cap = pl.env_rep_cap; ep.coarse = pl.env_coarse; ep.max_coarse = pl.env_max_coarse;
+            { LaunchTimer lt(h, PLOGP_KERNEL_ENVELOPE, st); CK(launch_envelope(ep, pl.env_threads, st)); }
+            g_launches += 1;
+        } else if (!pl.inline_sweep && pl.n_pairs > 0) {
             SweepParams sp{};
             sp.T = h->T; sp.G = pl.G;
             sp.pair_m = reinterpret_cast<const int32_t *>(h->d_grid + pl.off_pair_m);
@@ -426,6 +458,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             dp.n_mgroups = pl.dec_mgroups; dp.n_ptiles = pl.dec_ptiles; dp.mg = pl.dec_mg;
             dp.table0 = t0; dp.n_tables_launch = nt; dp.out_table0 = out.out_table0;
             dp.d_strategy = out.d_strategy; dp.d_sbytes = out.d_sbytes; dp.d_time = out.d_time;
+            dp.envelope = pl.envelope_short ? 1 : 0;
             dp.vec_out = (pl.G.n_m % 2 == 0) && pl.dec_mg >= 2 && reinterpret_cast<uintptr_t>(out.d_time) % 16 == 0 &&
                          reinterpret_cast<uintptr_t>(out.d_sbytes) % 8 == 0 && reinterpret_cast<uintptr_t>(out.d_strategy) % 2 == 0;
             { LaunchTimer lt(h, PLOGP_KERNEL_DECIDE, st); CK(launch_decide(dp, st)); }
@@ -457,8 +490,10 @@ extern "C" {
 
 // Validates host tables and lays them out as the kernels read them (key | gap | slope, padded).
 static int build_tables(int n_tables, int n_bp, int npad, const uint64_t *sizes_bytes, int sizes_shared,
-                        const double *gap, const double *latency, std::vector<double> &tab, std::vector<double> &lat)
+                        const double *gap, const double *latency, std::vector<double> &tab, std::vector<double> &lat,
+                        bool *monotone)
 {
+    *monotone = true;
     try {
         tab.assign(size_t(n_tables) * 3 * npad, 0.0);
         lat.assign(latency, latency + n_tables);
@@ -472,6 +507,7 @@ static int build_tables(int n_tables, int n_bp, int npad, const uint64_t *sizes_
         for (int i = 0; i < n_bp; ++i) {
             if (!std::isfinite(gp[i]) || gp[i] < 0.0) return PLOGP_E_INVAL;
             if (i && sz[i] <= sz[i - 1]) return PLOGP_E_INVAL;
+            if (i && gp[i] < gp[i - 1]) *monotone = false;
             if (double(sz[i]) >= kTwo53) return PLOGP_E_RANGE;
         }
         // Above the last size the last interval's line is continued: a falling line would turn g negative for
@@ -503,7 +539,8 @@ int plogp_table_load(int n_tables, int n_bp, const uint64_t *sizes_bytes, int si
     while (npad < n_bp) npad <<= 1;  // >= n_bp: at least one +inf key follows the last interval
 
     std::vector<double> tab, lat;
-    const int brc = build_tables(n_tables, n_bp, npad, sizes_bytes, sizes_shared, gap, latency, tab, lat);
+    bool monotone = false;
+    const int brc = build_tables(n_tables, n_bp, npad, sizes_bytes, sizes_shared, gap, latency, tab, lat, &monotone);
     if (brc != PLOGP_OK) return brc;
 
     plogp_tables *h = new (std::nothrow) plogp_tables();
@@ -526,6 +563,7 @@ int plogp_table_load(int n_tables, int n_bp, const uint64_t *sizes_bytes, int si
     h->T.n_tables = n_tables;
     h->T.n_bp = n_bp;
     h->T.npad = npad;
+    h->monotone = monotone;
     *out = h;
     return PLOGP_OK;
 }
@@ -538,8 +576,10 @@ int plogp_table_update(plogp_tables *h, const uint64_t *sizes_bytes, int sizes_s
     CK(cudaGetDevice(&dev));
     if (dev != h->device) return PLOGP_E_INVAL;
     std::vector<double> tab, lat;
-    const int brc = build_tables(h->T.n_tables, h->T.n_bp, h->T.npad, sizes_bytes, sizes_shared, gap, latency, tab, lat);
+    bool monotone = false;
+    const int brc = build_tables(h->T.n_tables, h->T.n_bp, h->T.npad, sizes_bytes, sizes_shared, gap, latency, tab, lat, &monotone);
     if (brc != PLOGP_OK) return brc;  // the tables on the device are untouched
+    h->monotone = monotone;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // pageable sources: the runtime stages them before returning, so the vectors may go out of scope
     CK(cudaMemcpyAsync(h->d_tab, tab.data(), tab.size() * sizeof(double), cudaMemcpyHostToDevice, st));

@@ -91,6 +91,8 @@ __device__ __forceinline__ void offer(double &bt, uint32_t &bcode, double t, uin
 
 }  // namespace
 
+// ENV: lower-envelope search (DecideParams::envelope), compiled apart so that the exhaustive kernel carries none of it.
+template <bool ENV>
 __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecideParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -156,8 +158,35 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
         const int ns = p.G.ns_of_m[midx];
         const int nsv = max(ns, 1);  // candidates actually evaluated (none fits: the whole message, k = 1)
         const double gm = sm.gm[mi];
-        const int o2 = n_un, o5 = o2 + (has2 ? nsv : 0), n1 = o5 + (has5 ? nsv : 0);
-        const int o9 = has7 ? 1 : 0, n2 = o9 + (has9 ? nsv : 0);
+        // Lower-envelope search (p.envelope, tables whose gaps never decrease): ids 2 and 9 keep only the candidate
+        // with the smallest g(s) k (their minimum over s for every P at once, a rounded fused multiply-add being
+        // monotone in it), id 5 only the candidates between its winners at the tile's last and first process
+        // count, one more on each side (the lines are sorted by slope g(s) + L, so the winner's index does not
+        // grow with P).  Otherwise every candidate enters the lists.
+        const bool env = ENV && ns > 0;
+        int q_c = 0, lo5 = 0, n5 = nsv;
+        if constexpr (ENV) if (env) {
+            const double x_first = sm.pm1[0], x_last = sm.pm1[n_valid - 1];
+            double qb = CUDART_INF, tf = CUDART_INF, tl = CUDART_INF;
+            int qc = kIntMax, ef = kIntMax, el = kIntMax;
+            for (int c = lane; c < ns; c += 32) {
+                const double gsv = sm.gs[c], k = static_cast<double>(segments(m_u, sm.sval[c], p.G.k_mode));
+                const double Q = gsv * k, B = gsv + L, C = gsv * (k - 1.0);
+                if (Q < qb) { qb = Q; qc = c; }
+                const double t1 = fma(x_first, B, C), t2 = fma(x_last, B, C);
+                if (t1 < tf) { tf = t1; ef = c; }
+                if (t2 < tl) { tl = t2; el = c; }
+            }
+            warp_min_pair(qb, qc);
+            warp_min_pair(tf, ef);
+            warp_min_pair(tl, el);
+            q_c = qc;
+            lo5 = max(min(ef, el) - 1, 0);
+            n5 = min(max(ef, el) + 1, ns - 1) - lo5 + 1;
+        }
+        const int nq = env ? 1 : nsv;  // entries of ids 2 and 9
+        const int o2 = n_un, o5 = o2 + (has2 ? nq : 0), n1 = o5 + (has5 ? n5 : 0);
+        const int o9 = has7 ? 1 : 0, n2 = o9 + (has9 ? nq : 0);
         const int n1p = round_up(n1, U), n2p = round_up(n2, U);
 
         // ---- the two lists of this message size, and each lane's best entry at the pilot's process count ----
@@ -202,21 +231,23 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 cand = static_cast<uint32_t>(c);
             }
             const double Q = gsv * k;
-            if (has2) {  // (P-1) (g(s) k) + L
-                l1[o2 + c] = make_double2(Q, L);
-                c1[o2 + c] = static_cast<uint16_t>((2u << 8) | cand);
-                pilot_offer(fma(x1_mid, Q, L), o2 + c);
+            const bool in_q = !env || c == q_c, in_5 = !env || (c >= lo5 && c < lo5 + n5);
+            const int pq = env ? 0 : c, p5 = env ? c - lo5 : c;  // positions inside the strategies' parts of the lists
+            if (has2 && in_q) {  // (P-1) (g(s) k) + L
+                l1[o2 + pq] = make_double2(Q, L);
+                c1[o2 + pq] = static_cast<uint16_t>((2u << 8) | cand);
+                pilot_offer(fma(x1_mid, Q, L), o2 + pq);
             }
-            if (has5) {  // (P-1) (g(s) + L) + g(s) (k-1)
+            if (has5 && in_5) {  // (P-1) (g(s) + L) + g(s) (k-1)
                 const double B = gsv + L, C = gsv * (k - 1.0);
-                l1[o5 + c] = make_double2(B, C);
-                c1[o5 + c] = static_cast<uint16_t>((5u << 8) | cand);
-                pilot_offer(fma(x1_mid, B, C), o5 + c);
+                l1[o5 + p5] = make_double2(B, C);
+                c1[o5 + p5] = static_cast<uint16_t>((5u << 8) | cand);
+                pilot_offer(fma(x1_mid, B, C), o5 + p5);
             }
-            if (has9) {  // floor(log2 P) g(s) k + ceil(log2 P) L
-                l2[o9 + c] = Q;
-                c2[o9 + c] = static_cast<uint16_t>((9u << 8) | cand);
-                pilot_offer(fma(x2_mid, Q, c2_mid), 256u + o9 + c);
+            if (has9 && in_q) {  // floor(log2 P) g(s) k + ceil(log2 P) L
+                l2[o9 + pq] = Q;
+                c2[o9 + pq] = static_cast<uint16_t>((9u << 8) | cand);
+                pilot_offer(fma(x2_mid, Q, c2_mid), 256u + o9 + pq);
             }
         }
         // warp-wide pilot: smallest time (high word first, then low word with the position in its last 9 bits)
@@ -393,17 +424,24 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
 
 size_t decide_smem_bytes(const TableDev &T, const GridDev &G) { return dec_layout(T.npad, G.n_s, nullptr, nullptr); }
 
+template <bool ENV>
+static cudaError_t launch_decide_t(const DecideParams &p, size_t smem, unsigned blocks, cudaStream_t st)
+{
+    cudaError_t e = cudaSuccess;
+    if (smem > 48 * 1024)
+        e = cudaFuncSetAttribute(decide_kernel<ENV>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    decide_kernel<ENV><<<blocks, kDecThreads, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_decide(const DecideParams &p, cudaStream_t st)
 {
     const size_t smem = decide_smem_bytes(p.T, p.G);
-    cudaError_t e = cudaSuccess;
-    if (smem > 48 * 1024)
-        e = cudaFuncSetAttribute(decide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
     const long long blocks = static_cast<long long>(p.n_mgroups) * p.n_ptiles * p.n_tables_launch;
     if (blocks <= 0 || blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    decide_kernel<<<static_cast<unsigned>(blocks), kDecThreads, smem, st>>>(p);
-    return cudaGetLastError();
+    return p.envelope ? launch_decide_t<true>(p, smem, static_cast<unsigned>(blocks), st)
+                      : launch_decide_t<false>(p, smem, static_cast<unsigned>(blocks), st);
 }
 
 }  // namespace plogp

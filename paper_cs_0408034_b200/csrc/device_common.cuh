@@ -107,12 +107,23 @@ struct GapWalk {
     }
 };
 
+// Lexicographic minimum of (t, e) over a warp (all lanes receive it).
+__device__ __forceinline__ void warp_min_pair(double &t, int &e)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const double t2 = __shfl_xor_sync(0xffffffffu, t, off);
+        const int e2 = __shfl_xor_sync(0xffffffffu, e, off);
+        if (t2 < t || (t2 == t && e2 < e)) { t = t2; e = e2; }
+    }
+}
+
 // Sum of g(j m) for j = jlo .. jhi (jlo <= jhi) in closed form: inside one table interval g is a line, so the
 // terms whose arguments fall into it are an arithmetic series, n gap_i + slope_i (m (jlo' + jhi') n / 2 - n key_i);
 // the loop runs over the table intervals that the arguments cross (at most n_bp), not over j.  Below the first
 // size g is constant (its first value), above the last size the last interval's line goes on.  This is what
 // keeps a gap in a process-count list, or a first process count far above 2, from turning into a long loop.
-__device__ __forceinline__ double chain_range_sum(const double *s_tab, int npad, double md, long long jlo, long long jhi)
+static __device__ __noinline__ double chain_range_sum(const double *s_tab, int npad, double md, long long jlo, long long jhi)
 {
     double sum = 0.0;
     long long j = jlo;

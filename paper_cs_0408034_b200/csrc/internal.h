@@ -48,6 +48,20 @@ struct SweepParams {
     int table0;          // first table of this launch (blockIdx.y is relative to it)
 };
 
+// Envelope kernel (exact fast path of the segment-size search): same scratch layout as the sweep kernel with
+// one row per message size.
+struct EnvParams {
+    TableDev T;
+    GridDev G;
+    int table0, n_tables_launch;
+    double *part_time;   // [n_tables_batch][n_seg][n_m][n_P]
+    uint32_t *part_idx;  // same shape: index of s in the candidate list
+    int n_seg;
+    int rep_cap;     // entries of the shared-memory list of representatives (longer lists go through it in windows)
+    int coarse;      // distance between the coarse process-count indices
+    int max_coarse;  // capacity of the coarse-winner array (>= number of coarse indices)
+};
+
 struct FusedParams {
     TableDev T;
     GridDev G;
@@ -83,6 +97,7 @@ struct DecideParams {
     GridDev G;
     int n_mgroups, n_ptiles;
     int mg;  // message sizes per CTA, 1..kDecMG
+    int envelope;  // lower-envelope search: the lists keep only the candidates that can win (see decide.cu)
     int vec_out;  // outputs aligned for two message sizes per store (n_m even, 16 / 8 / 2-byte aligned bases)
     int table0, n_tables_launch;
     int out_table0;  // table whose results sit at the start of the output arrays
@@ -114,5 +129,7 @@ cudaError_t launch_s1_tiles(const S1Params &p, cudaStream_t st);
 size_t decide_smem_bytes(const TableDev &T, const GridDev &G);
 cudaError_t launch_decide(const DecideParams &p, cudaStream_t st);
 cudaError_t launch_fp64_probe(double *d_sink, int iters, int blocks, cudaStream_t st);
+size_t envelope_smem_bytes(const TableDev &T, int threads, int rep_cap, int max_coarse);
+cudaError_t launch_envelope(const EnvParams &p, int threads, cudaStream_t st);
 
 }  // namespace plogp

@@ -269,7 +269,7 @@ size_t fused_smem_bytes(const TableDev &T, const GridDev &G, bool inline_sweep)
 }
 
 template <bool PREDICT>
-__global__ void __launch_bounds__(kThreads) fused_kernel(const FusedParams p)
+__global__ void __launch_bounds__(kThreads, 2) fused_kernel(const FusedParams p)
 {
     constexpr int R = kFusedR;
     extern __shared__ __align__(16) unsigned char smem_raw[];

@@ -31,7 +31,8 @@ class Grid(C.Structure):
                 ("m", C.POINTER(C.c_uint64)), ("n_m", C.c_int32),
                 ("s", C.POINTER(C.c_uint64)), ("n_s", C.c_int64),
                 ("s_lo", C.c_uint64), ("s_hi", C.c_uint64), ("s_step", C.c_uint64),
-                ("dtype_bytes", C.c_uint32), ("strategy_mask", C.c_uint32), ("k_mode", C.c_int32)]
+                ("dtype_bytes", C.c_uint32), ("strategy_mask", C.c_uint32), ("k_mode", C.c_int32),
+                ("search_mode", C.c_int32)]
 
 
 if not os.path.exists(LIB_PATH):
@@ -152,7 +153,7 @@ class GridArgs:
     """Keeps the host arrays of a ``plogp_grid`` alive next to the struct."""
 
     def __init__(self, m, P=None, P_lo=2, P_hi=2, s=None, s_lo=0, s_hi=0, s_step=0,
-                 dtype_bytes=4, strategy_mask=(1 << 13) - 1, k_mode=0):
+                 dtype_bytes=4, strategy_mask=(1 << 13) - 1, k_mode=0, search_mode=0):
         self.m = np.ascontiguousarray(m, dtype=np.uint64)
         self.P = None if P is None else np.ascontiguousarray(P, dtype=np.int32)
         self.s = None if s is None else np.ascontiguousarray(s, dtype=np.uint64)
@@ -168,12 +169,13 @@ class GridArgs:
             g.n_s = len(self.s)
         g.s_lo, g.s_hi, g.s_step = int(s_lo), int(s_hi), int(s_step)
         g.dtype_bytes, g.strategy_mask, g.k_mode = int(dtype_bytes), int(strategy_mask), int(k_mode)
+        g.search_mode = int(search_mode)
         self.struct = g
 
     @classmethod
     def from_workload(cls, w) -> "GridArgs":
         return cls(w.m, getattr(w, "P_list", None), w.P_lo, w.P_hi, w.s_list, w.s_lo, w.s_hi, w.s_step, w.dtype_bytes,
-                   w.strategy_mask, w.k_mode)
+                   w.strategy_mask, w.k_mode, getattr(w, "search_mode", 0))
 
     @property
     def n_P(self) -> int:
@@ -270,7 +272,7 @@ def scatter_chain_static(d_sizes, d_gap, latency: float, P_lo: int, P_hi: int, d
     return out
 
 
-KERNEL_KINDS = ("sweep_kernel", "s1_tile_sum_kernel", "fused_kernel", "decide_kernel", "scatter_kernel")
+KERNEL_KINDS = ("sweep_kernel", "s1_tile_sum_kernel", "fused_kernel", "decide_kernel", "scatter_kernel", "envelope_kernel")
 
 
 def profile_enable(tables: Tables, enable: bool = True) -> None:

@@ -83,6 +83,7 @@ class Workload:
     seed: int = 0
     notes: dict = field(default_factory=dict)
     P_list: Optional[np.ndarray] = None   # int32 ascending process counts; None => P_lo..P_hi
+    search_mode: int = 0                  # 0 = exhaustive segment search, 1 = lower envelope (same results)
 
     @property
     def n_tables(self) -> int:

@@ -327,3 +327,95 @@ def test_scatter_chain_with_a_far_first_process_count_and_wide_gaps(plogp):
     run_both(plogp, replace(base, P_lo=2, P_hi=int(P[-1]), P_list=P))
     # the same through the general kernel (Broadcast strategies enabled as well)
     run_both(plogp, replace(wl.config2(P_hi=40, n_m=20, n_s=9), P_lo=3000, P_hi=3040))
+
+
+# ---- search_mode 1: the segment-size search by lower envelope (same results as the exhaustive search) ----
+
+def _envelope(w):
+    from dataclasses import replace
+    return replace(w, search_mode=1)
+
+
+def test_envelope_search_on_short_and_long_candidate_lists(plogp):
+    from dataclasses import replace
+    run_both(plogp, _envelope(wl.config1()))
+    run_both(plogp, _envelope(replace(wl.config1(), strategy_mask=wl.ALL_STRATEGIES, k_mode=1)))
+    run_both(plogp, _envelope(wl.config2(P_hi=300, n_m=45, n_s=29)))
+    run_both(plogp, _envelope(wl.config4(n_tables=6)), tables=[0, 3, 5], p_idx=np.r_[0:70, 250:260, 500:511])
+    # long lists: every multiple of 4 B (16384 candidates), all three segmented strategies, both k modes
+    w = replace(wl.config3(P_hi=700, n_m=6, m_lo=1 << 10, m_hi=1 << 16, s_hi=1 << 14), strategy_mask=wl.ALL_STRATEGIES)
+    run_both(plogp, _envelope(w), p_idx=np.r_[0:50, 250:270, 500:520, 690:699])
+    run_both(plogp, _envelope(replace(w, k_mode=1)), p_idx=np.r_[0:50, 250:270, 500:520, 690:699])
+    for mask in (1 << 2, 1 << 5, 1 << 9, (1 << 2) | (1 << 9), (1 << 5) | (1 << 9)):
+        run_both(plogp, _envelope(replace(w, strategy_mask=mask, P_hi=130)))
+
+
+def test_envelope_search_with_more_representatives_than_fit_in_shared_memory(plogp):
+    """m = 48 MB with every multiple of 4 B up to 1 MB as candidates: more than 6144 distinct segment counts, so
+    the list of representatives goes through shared memory in several windows."""
+    from dataclasses import replace
+    w = replace(wl.config3(P_hi=600, n_m=2, m_lo=48 << 20, m_hi=49 << 20), search_mode=1)
+    k = -(-int(w.m[0]) // np.arange(4, (1 << 20) + 1, 4))
+    assert len(np.unique(k)) > 6144
+    run_both(plogp, w, p_idx=np.r_[0:40, 100:110, 300:340, 590:599])
+
+
+def test_envelope_search_on_a_table_with_a_dip_takes_the_exhaustive_search(plogp):
+    """A table whose gap decreases somewhere does not qualify for the envelope search; the call must still
+    return the exhaustive result."""
+    import torch
+    w = wl.config2(P_hi=120, n_m=30, n_s=20)
+    gaps = w.gaps.copy()
+    gaps[0, 7] = gaps[0, 6] * 0.9   # a dip in the middle; the last interval still rises
+    from dataclasses import replace
+    run_both(plogp, replace(w, gaps=gaps, search_mode=1))
+
+
+def test_envelope_search_reproduces_exact_ties(plogp):
+    """The flat table of the exact-tie test: with search_mode 1 the picks must equal the exhaustive ones bit for bit."""
+    import torch
+    sizes = np.array([4, 64, 1024, 1 << 20], dtype=np.uint64)
+    gaps = np.ones((1, 4))
+    lat = np.array([2.0])
+    m = np.array([8, 100, 1000, 4096, 10000, 65536, 100000], dtype=np.uint64)
+    P = np.arange(2, 140, dtype=np.int32)
+    for s_kw in (dict(s=wl.log_spaced_multiples(4, 1 << 16, 40)), dict(s=None, s_lo=4, s_hi=4096, s_step=4)):
+        with plogp.Tables(sizes, gaps, lat) as tabs:
+            a = plogp.select_best(tabs, plogp.GridArgs(m, P=P, **s_kw))
+            b = plogp.select_best(tabs, plogp.GridArgs(m, P=P, search_mode=1, **s_kw))
+            pa = plogp.predict(tabs, plogp.GridArgs(m, P=P, **s_kw))
+            pb = plogp.predict(tabs, plogp.GridArgs(m, P=P, search_mode=1, **s_kw))
+            torch.cuda.synchronize()
+        assert torch.equal(a.strategy, b.strategy) and torch.equal(a.s_bytes, b.s_bytes)
+        assert torch.equal(a.time.view(torch.int64), b.time.view(torch.int64))
+        assert torch.equal(pa.best_s, pb.best_s) and torch.equal(pa.time.view(torch.int64), pb.time.view(torch.int64))
+
+
+def test_envelope_search_at_full_size(plogp):
+    """The exhaustive-sweep configuration (262144 candidates, P up to 4096) and the batched one (4096 tables)
+    through the envelope search: sampled cells against the oracle, everything else against the exhaustive path."""
+    import torch
+    w = wl.config3()
+    ot = oracle_tables(w)
+    p_idx = np.unique(np.r_[[0, 1, 2, 63, 64, 65, 255, 256, 2047, 2048, 4093, 4094], (wl.uniform(w.seed, 5100 + np.arange(30)) * w.n_P).astype(np.int64)])
+    m_idx = np.unique(np.r_[[0, 1, 64, 127], (wl.uniform(w.seed, 6100 + np.arange(12)) * w.n_m).astype(np.int64)])
+    with plogp.Tables.from_workload(w) as tabs:
+        ex = plogp.select_best(tabs, w)
+        env = plogp.select_best(tabs, _envelope(w))
+        torch.cuda.synchronize()
+        assert check_decision(w, ot, env, p_idx=p_idx, m_idx=m_idx) > 0
+    same = (ex.strategy == env.strategy) & (ex.s_bytes == env.s_bytes)
+    # wherever the picks differ the two times must agree to 1e-9 (ties inside the margin)
+    rel = ((ex.time - env.time).abs() / ex.time)[:, 0]
+    assert float(rel.max()) <= 1e-9
+    assert float(same[:, 0].float().mean()) > 0.999
+    w4 = wl.config4()
+    with plogp.Tables.from_workload(w4) as tabs:
+        env = plogp.select_best(tabs, _envelope(w4))
+        torch.cuda.synchronize()
+        k = 20000
+        c = np.arange(k)
+        t_idx = (wl.uniform(w4.seed, 7_500_000 + c) * w4.n_tables).astype(np.int64)
+        pi = (wl.uniform(w4.seed, 8_500_000 + c) * w4.n_P).astype(np.int64)
+        mi = (wl.uniform(w4.seed, 9_500_000 + c) * w4.n_m).astype(np.int64)
+        assert check_decision_cells(w4, env, t_idx, pi, mi) == 2 * k
