@@ -258,6 +258,38 @@ void po_select_grid(uint32_t mask, int n_P, int n_m, const double *time, const u
     }
 }
 
+/* ---- Sensitivity to the segment size ---- */
+uint64_t po_effective_segment(uint64_t m, uint64_t s_fixed) { return s_fixed <= m ? s_fixed : m; }
+
+void po_surface_grid(const po_table *t, uint32_t mask, const int64_t *P, int n_P, const uint64_t *m, int n_m,
+                     const po_sgrid *sg, int k_mode, double *out)
+{
+    static const int seg_ids[PO_N_SEGMENTED] = {2, 5, 9};
+    const int64_t n_s = sgrid_count(sg);
+    for (int q = 0; q < PO_N_SEGMENTED; ++q)
+        for (int ip = 0; ip < n_P; ++ip)
+            for (int im = 0; im < n_m; ++im)
+                for (int64_t is = 0; is < n_s; ++is) {
+                    uint64_t s = sgrid_at(sg, is);
+                    double v = NAN;
+                    if (((mask >> seg_ids[q]) & 1u) && s <= m[im]) v = po_model(t, seg_ids[q], P[ip], m[im], s, k_mode);
+                    out[(((size_t)q * n_P + ip) * n_m + im) * (size_t)n_s + (size_t)is] = v;
+                }
+}
+
+void po_fixed_segment_grid(const po_table *t, uint32_t mask, const int64_t *P, int n_P, const uint64_t *m,
+                           int n_m, uint64_t s_fixed, int k_mode, double *time_fixed)
+{
+    static const int seg_ids[PO_N_SEGMENTED] = {2, 5, 9};
+    for (int q = 0; q < PO_N_SEGMENTED; ++q) {
+        if (!((mask >> seg_ids[q]) & 1u)) continue;
+        for (int ip = 0; ip < n_P; ++ip)
+            for (int im = 0; im < n_m; ++im)
+                time_fixed[((size_t)q * n_P + ip) * n_m + im] =
+                    po_model(t, seg_ids[q], P[ip], m[im], po_effective_segment(m[im], s_fixed), k_mode);
+    }
+}
+
 int po_threads(void)
 {
 #ifdef _OPENMP

@@ -106,6 +106,22 @@ void po_predict_grid(const po_table *t, uint32_t mask, const int64_t *P, int n_P
 void po_select_grid(uint32_t mask, int n_P, int n_m, const double *time, const uint64_t *best_s,
                     uint8_t *strategy, uint64_t *s_out, double *time_out, double *runner_up);
 
+/* ---- Sensitivity to the segment size (Section 3.1; the measured Segmented Chain of Fig. 1(b) used 8 kB) ----
+ *
+ * The segment size a fixed setting really uses for a message m: s_fixed itself when it fits (s_fixed <= m),
+ * otherwise the whole message (s = m, one segment), as Section 3.1 sends smaller messages unsegmented. */
+uint64_t po_effective_segment(uint64_t m, uint64_t s_fixed);
+
+/* Model surface over s: out[q][ip][im][is] = po_model(id_q, P[ip], m[im], s_is) for the segmented ids
+ * q = 0,1,2 (2, 5, 9) enabled in mask and every candidate s_is of the grid; NaN where s_is > m[im]
+ * (not a candidate for that message) or the id is disabled.  n_s = number of candidates of sg. */
+void po_surface_grid(const po_table *t, uint32_t mask, const int64_t *P, int n_P, const uint64_t *m, int n_m,
+                     const po_sgrid *sg, int k_mode, double *out);
+
+/* time_fixed[q][ip][im] = po_model(id_q, P, m, po_effective_segment(m, s_fixed)); disabled ids untouched. */
+void po_fixed_segment_grid(const po_table *t, uint32_t mask, const int64_t *P, int n_P, const uint64_t *m,
+                           int n_m, uint64_t s_fixed, int k_mode, double *time_fixed);
+
 int po_threads(void);
 
 #ifdef __cplusplus

@@ -82,6 +82,13 @@ def _load():
         lib.po_select_grid.restype = None
         lib.po_select_grid.argtypes = [C.c_uint32, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.po_effective_segment.restype = C.c_uint64
+        lib.po_effective_segment.argtypes = [C.c_uint64, C.c_uint64]
+        lib.po_surface_grid.restype = None
+        lib.po_surface_grid.argtypes = [TP, C.c_uint32, C.c_void_p, C.c_int, C.c_void_p, C.c_int, SP, C.c_int, C.c_void_p]
+        lib.po_fixed_segment_grid.restype = None
+        lib.po_fixed_segment_grid.argtypes = [TP, C.c_uint32, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_uint64,
+                                              C.c_int, C.c_void_p]
         lib.po_threads.restype = C.c_int
         _lib = lib
     return _lib
@@ -197,3 +204,45 @@ def select_grid(mask: int, pred: Predicted) -> Decision:
     _load().po_select_grid(int(mask), nP, nm, pred.time.ctypes.data, pred.best_s.ctypes.data,
                            strategy.ctypes.data, s.ctypes.data, time.ctypes.data, ru.ctypes.data)
     return Decision(strategy, s, time, ru)
+
+
+def n_candidates(sg: SGrid) -> int:
+    if sg.values is not None:
+        return len(sg.values)
+    c = sg._c
+    return 0 if c.step == 0 or c.hi < c.lo else int((c.hi - c.lo) // c.step) + 1
+
+
+def surface_grid(t: Table, mask: int, P, m, sg: SGrid, k_mode: int = 0) -> np.ndarray:
+    """Model surface over s: [3][n_P][n_m][n_s] for ids 2, 5, 9 (NaN where s > m or the id is disabled)."""
+    P = np.ascontiguousarray(P, dtype=np.int64)
+    m = np.ascontiguousarray(m, dtype=np.uint64)
+    out = np.full((3, len(P), len(m), n_candidates(sg)), np.nan, dtype=np.float64)
+    _load().po_surface_grid(t.ref, int(mask), P.ctypes.data, len(P), m.ctypes.data, len(m), sg.ref, int(k_mode),
+                            out.ctypes.data)
+    return out
+
+
+def fixed_segment_grid(t: Table, mask: int, P, m, s_fixed: int, k_mode: int = 0) -> np.ndarray:
+    """Times of ids 2, 5, 9 with one fixed segment size (the whole message where it does not fit): [3][n_P][n_m]."""
+    P = np.ascontiguousarray(P, dtype=np.int64)
+    m = np.ascontiguousarray(m, dtype=np.uint64)
+    out = np.full((3, len(P), len(m)), np.nan, dtype=np.float64)
+    _load().po_fixed_segment_grid(t.ref, int(mask), P.ctypes.data, len(P), m.ctypes.data, len(m), int(s_fixed),
+                                  int(k_mode), out.ctypes.data)
+    return out
+
+
+def effective_segment(m: int, s_fixed: int) -> int:
+    return _load().po_effective_segment(int(m), int(s_fixed))
+
+
+def decision_boundaries(strategy: np.ndarray) -> np.ndarray:
+    """Where the selected strategy changes in the (P, m) plane: for strategy[..., n_P, n_m] returns uint8 flags of
+    the same shape, bit 0 = differs from the next larger P (same m), bit 1 = differs from the next larger m
+    (same P); the last row / column has no such neighbour and gets 0 there."""
+    s = np.asarray(strategy)
+    out = np.zeros(s.shape, dtype=np.uint8)
+    out[..., :-1, :] |= (s[..., :-1, :] != s[..., 1:, :]).astype(np.uint8)
+    out[..., :, :-1] |= ((s[..., :, :-1] != s[..., :, 1:]).astype(np.uint8) << 1)
+    return out
