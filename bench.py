@@ -362,6 +362,67 @@ class Bench:
         ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / steps, self.world, "cuda")
         return ms, h2d, d2h
 
+    def time_aux(self, name, w, fn, nbytes, steps=10, warmup=3):
+        """Times one streaming call (CUDA events on the launching stream, L2 flushed between steps when the
+        call moves less than 256 MB) and reports it against the HBM roofline of its algorithmic bytes."""
+        torch = self.torch
+        if self.flush_buf is None:
+            self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        flush = nbytes < (256 << 20)
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        ms = 0.0
+        for _ in range(steps):
+            if flush:
+                self.flush_buf.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            b.synchronize()
+            ms += a.elapsed_time(b)
+        ms /= steps
+        return {"call": name, "config": {"workload": w.name, "tables_per_gpu": w.n_tables, "P": [w.P_lo, w.P_hi], "n_m": w.n_m,
+                                         "n_s": int(len(w.s_values()))},
+                "steps": steps, "ms_per_step": ms,
+                "roofline": {"bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": self.hbm_gbs, "unit": "GB/s",
+                             "frac": nbytes / (self.hbm_gbs * 1e9) / (ms * 1e-3), "algorithmic_bytes": nbytes,
+                             "peak_source": "HBM copy bandwidth, of %s" % self.peak_src}}
+
+    def aux_entries(self, w4):
+        """The segment-size sensitivity calls: the model surface over s on the dense single-table grid, the fixed
+        8 kB segment size and the decision boundaries on the batched workload."""
+        plogp, torch = self.plogp, self.torch
+        out = []
+        w2 = wl.config2()
+        with plogp.Tables.from_workload(w2) as tabs:
+            g = plogp.GridArgs.from_workload(w2)
+            surf = plogp.segment_surface(tabs, g)
+            out.append(self.time_aux("plogp_segment_surface", w2, lambda: plogp.segment_surface(tabs, g, out=surf), surf.numel() * 8))
+            del surf
+        with plogp.Tables.from_workload(w4) as tabs:
+            g = plogp.GridArgs.from_workload(w4)
+            pred = plogp.predict(tabs, g)
+            cells = w4.n_tables * w4.n_P * w4.n_m
+            shape = (w4.n_tables, 3, w4.n_P, w4.n_m)
+            fixed = torch.empty(shape, dtype=torch.float64, device="cuda")
+            ratio = torch.empty(shape, dtype=torch.float64, device="cuda")
+
+            def sens():
+                plogp._check(plogp.lib.plogp_segment_sensitivity(tabs.handle, g.ref, 8192, pred.time.data_ptr(), fixed.data_ptr(),
+                                                                 ratio.data_ptr(), plogp._stream_ptr(None)), "plogp_segment_sensitivity")
+            out.append(self.time_aux("plogp_segment_sensitivity (s = 8192 B)", w4, sens, 3 * cells * 8 * 3))
+            del pred, fixed, ratio
+            dec = plogp.select_best(tabs, g)
+            bnd = torch.empty_like(dec.strategy)
+
+            def bounds():
+                plogp._check(plogp.lib.plogp_decision_boundaries(w4.n_tables, w4.n_P, w4.n_m, dec.strategy.data_ptr(), bnd.data_ptr(),
+                                                                 plogp._stream_ptr(None)), "plogp_decision_boundaries")
+            out.append(self.time_aux("plogp_decision_boundaries", w4, bounds, 2 * cells * 2))
+        return out
+
     def rooflines(self, m):
         """Per-kernel roofline objects of one measurement, the dominant kernel's copy and the whole-step figure."""
         if self.fma_rate is None:
@@ -505,6 +566,7 @@ def run_ours(args, rank, local_rank, world):
             others.append(b.entry(mm, note="segment search by lower envelope (search_mode 1): same decision table, "
                                            "skipped cells are not counted as model cells"))
         line["workloads"] = others
+        line["sensitivity_calls"] = b.aux_entries(w)
     if world == 1 and not args.no_cpu_baseline:
         v, cores, text = oracle_sample_rate(w, 15.0)
         v1, _, text1 = oracle_sample_rate(w, 8.0, threads=1)

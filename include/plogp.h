@@ -161,6 +161,42 @@ int plogp_select_best(plogp_tables *tables, const plogp_grid *grid, uint8_t *d_s
 int plogp_select_best_host(plogp_tables *tables, const plogp_grid *grid, uint8_t *h_strategy,
                            uint32_t *h_s_bytes, double *h_time, void *stream);
 
+/*
+ * Model surface over the segment size (Section 3.1 searches the s that minimises these values): the models of the
+ * segmented strategies (ids 2, 5, 9 of Table 1, in this order) for every candidate s of the grid.
+ *   d_surface  DEVICE, double [n_tables][3][n_P][n_m][n_s], s fastest, n_s = number of candidates of the grid;
+ *              NaN where s > m (not a candidate for that message); planes of disabled ids are left untouched.
+ * The caller sizes the grid so that the surface fits.  Same stream and ownership rules as plogp_predict.
+ */
+int plogp_segment_surface(plogp_tables *tables, const plogp_grid *grid, double *d_surface, void *stream);
+
+/*
+ * What one fixed segment size costs (the measured Segmented Chain of the paper's Fig. 1(b) used 8 kB segments for
+ * every message; Section 3.1 tunes the size instead).  For every table, segmented strategy (ids 2, 5, 9), P and m:
+ *   d_time_fixed  DEVICE, double [n_tables][3][n_P][n_m]: the model with s = s_fixed, or with the whole message as
+ *                 its one segment (s = m, k = 1) where s_fixed > m, as Section 3.1 sends smaller messages unsegmented
+ *   d_ratio       DEVICE, double [n_tables][3][n_P][n_m]: d_time_fixed divided by the minimum over the grid's
+ *                 candidates, read from d_pred_time; >= 1 wherever s_fixed is itself a candidate.  May be NULL,
+ *                 together with d_pred_time.
+ *   d_pred_time   DEVICE, the d_time output of plogp_predict for the same tables and the same grid
+ *                 ([n_tables][13][n_P][n_m]); only the planes of the enabled segmented ids are read.
+ *   s_fixed       bytes, a positive multiple of grid->dtype_bytes, < 2^32; it need not be one of the grid's candidates.
+ * Planes of disabled ids are left untouched.
+ */
+int plogp_segment_sensitivity(plogp_tables *tables, const plogp_grid *grid, uint64_t s_fixed, const double *d_pred_time,
+                              double *d_time_fixed, double *d_ratio, void *stream);
+
+/*
+ * Decision boundaries in the (P, m) plane (Sections 1 and 5: the tuner's result is a map from parameter sets to
+ * strategies; this marks where the map changes).
+ *   d_strategy  DEVICE, uint8 [n_tables][2][n_P][n_m], the d_strategy output of plogp_select_best
+ *   d_boundary  DEVICE, uint8 [n_tables][2][n_P][n_m]: bit 0 set where the next larger process count (same m) has
+ *               another strategy, bit 1 where the next larger message size (same P) has; the last row / column
+ *               has no such neighbour.
+ * Needs no table handle: it only reads the decision table.
+ */
+int plogp_decision_boundaries(int n_tables, int n_P, int n_m, const uint8_t *d_strategy, uint8_t *d_boundary, void *stream);
+
 /* Static description of a status code. */
 const char *plogp_status_string(int status);
 

@@ -729,6 +729,72 @@ int plogp_select_best_host(plogp_tables *h, const plogp_grid *grid, uint8_t *h_s
     return PLOGP_OK;
 }
 
+int plogp_segment_surface(plogp_tables *h, const plogp_grid *grid, double *d_surface, void *stream)
+{
+    if (!h || !grid || !d_surface) return PLOGP_E_INVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev != h->device) return PLOGP_E_INVAL;
+    int rc = prepare(h, grid, st);
+    if (rc != PLOGP_OK) { h->plan = Plan(); return rc; }
+    const Plan &pl = h->plan;
+    if (pl.empty || pl.n_seg == 0 || pl.G.n_s == 0) return PLOGP_OK;
+    for (int t0 = 0; t0 < h->T.n_tables; t0 += 65535) {
+        SensParams sp{};
+        sp.T = h->T; sp.G = pl.G;
+        sp.table0 = t0; sp.n_tables_launch = std::min(65535, h->T.n_tables - t0); sp.out_table0 = 0;
+        sp.surface = d_surface;
+        CK(launch_surface(sp, st));
+        g_launches += 1;
+    }
+    return PLOGP_OK;
+}
+
+int plogp_segment_sensitivity(plogp_tables *h, const plogp_grid *grid, uint64_t s_fixed, const double *d_pred_time,
+                              double *d_time_fixed, double *d_ratio, void *stream)
+{
+    if (!h || !grid || !d_time_fixed) return PLOGP_E_INVAL;
+    if ((d_ratio == nullptr) != (d_pred_time == nullptr)) return PLOGP_E_INVAL;
+    if (s_fixed == 0 || grid->dtype_bytes == 0 || s_fixed % grid->dtype_bytes) return PLOGP_E_INVAL;
+    if (s_fixed >= kTwo32) return PLOGP_E_RANGE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev != h->device) return PLOGP_E_INVAL;
+    int rc = prepare(h, grid, st);
+    if (rc != PLOGP_OK) { h->plan = Plan(); return rc; }
+    const Plan &pl = h->plan;
+    if (pl.empty || pl.n_seg == 0) return PLOGP_OK;
+    // enough CTAs to fill the GPU, each with a run of process counts per warp
+    const long long base_blocks = (long long)((pl.G.n_m + 31) / 32) * h->T.n_tables;
+    int p_per_cta = pl.G.n_P;
+    while (p_per_cta > 8 && base_blocks * ((pl.G.n_P + p_per_cta - 1) / p_per_cta) < (long long)h->sm_count * 8) p_per_cta = (p_per_cta + 1) / 2;
+    for (int t0 = 0; t0 < h->T.n_tables; t0 += 65535) {
+        SensParams sp{};
+        sp.T = h->T; sp.G = pl.G;
+        sp.table0 = t0; sp.n_tables_launch = std::min(65535, h->T.n_tables - t0); sp.out_table0 = 0;
+        sp.s_fixed = uint32_t(s_fixed); sp.p_per_cta = p_per_cta;
+        sp.pred_time = d_pred_time; sp.time_fixed = d_time_fixed; sp.ratio = d_ratio;
+        CK(launch_fixed(sp, st));
+        g_launches += 1;
+    }
+    return PLOGP_OK;
+}
+
+int plogp_decision_boundaries(int n_tables, int n_P, int n_m, const uint8_t *d_strategy, uint8_t *d_boundary, void *stream)
+{
+    if (n_tables < 0 || n_P < 0 || n_m < 0) return PLOGP_E_INVAL;
+    if (n_tables == 0 || n_P == 0 || n_m == 0) return PLOGP_OK;
+    if (!d_strategy || !d_boundary) return PLOGP_E_INVAL;
+    int dev = 0, sms = 0;
+    CK(cudaGetDevice(&dev));
+    CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CK(launch_boundaries(d_strategy, d_boundary, 2LL * n_tables, n_P, n_m, sms, static_cast<cudaStream_t>(stream)));
+    g_launches += 1;
+    return PLOGP_OK;
+}
+
 const char *plogp_status_string(int status)
 {
     switch (status) {

@@ -62,6 +62,18 @@ struct EnvParams {
     int max_coarse;  // capacity of the coarse-winner array (>= number of coarse indices)
 };
 
+// Segment-size sensitivity kernels (sensitivity.cu)
+struct SensParams {
+    TableDev T;
+    GridDev G;
+    int table0, n_tables_launch, out_table0;
+    double *surface;           // [n_tables][3][n_P][n_m][n_s]
+    uint32_t s_fixed;          // the fixed segment size (fixed_kernel)
+    int p_per_cta;             // process counts per CTA (fixed_kernel)
+    const double *pred_time;   // [n_tables][13][n_P][n_m] from plogp_predict, or nullptr together with ratio
+    double *time_fixed, *ratio;  // [n_tables][3][n_P][n_m]
+};
+
 struct FusedParams {
     TableDev T;
     GridDev G;
@@ -129,6 +141,9 @@ cudaError_t launch_s1_tiles(const S1Params &p, cudaStream_t st);
 size_t decide_smem_bytes(const TableDev &T, const GridDev &G);
 cudaError_t launch_decide(const DecideParams &p, cudaStream_t st);
 cudaError_t launch_fp64_probe(double *d_sink, int iters, int blocks, cudaStream_t st);
+cudaError_t launch_surface(const SensParams &p, cudaStream_t st);
+cudaError_t launch_fixed(const SensParams &p, cudaStream_t st);
+cudaError_t launch_boundaries(const uint8_t *d_strategy, uint8_t *d_boundary, long long n_planes, int n_P, int n_m, int sm_count, cudaStream_t st);
 size_t envelope_smem_bytes(const TableDev &T, int threads, int rep_cap, int max_coarse);
 cudaError_t launch_envelope(const EnvParams &p, int threads, cudaStream_t st);
 

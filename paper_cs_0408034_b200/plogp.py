@@ -20,7 +20,7 @@ N_STRATEGIES = 13
 SEGMENTED_IDS = (2, 5, 9)
 EXPORTS = ("plogp_table_load", "plogp_table_update", "plogp_table_free", "plogp_predict", "plogp_select_best", "plogp_select_best_host",
            "plogp_status_string", "plogp_last_cuda_error", "plogp_kernel_launches", "plogp_fp64_fma_rate", "plogp_profile_enable", "plogp_profile_read",
-           "plogp_scatter_chain_static")
+           "plogp_scatter_chain_static", "plogp_segment_surface", "plogp_segment_sensitivity", "plogp_decision_boundaries")
 
 OK, E_INVAL, E_NOMEM, E_CUDA, E_RANGE = 0, -1, -2, -3, -4
 
@@ -63,6 +63,12 @@ lib.plogp_last_cuda_error.argtypes = []
 lib.plogp_scatter_chain_static.restype = C.c_int
 lib.plogp_scatter_chain_static.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_double, C.c_int32, C.c_int32,
                                            C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+lib.plogp_segment_surface.restype = C.c_int
+lib.plogp_segment_surface.argtypes = [C.c_void_p, C.POINTER(Grid), C.c_void_p, C.c_void_p]
+lib.plogp_segment_sensitivity.restype = C.c_int
+lib.plogp_segment_sensitivity.argtypes = [C.c_void_p, C.POINTER(Grid), C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+lib.plogp_decision_boundaries.restype = C.c_int
+lib.plogp_decision_boundaries.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.plogp_profile_enable.restype = C.c_int
 lib.plogp_profile_enable.argtypes = [C.c_void_p, C.c_int]
 lib.plogp_profile_read.restype = C.c_int
@@ -304,4 +310,47 @@ def select_best_host(tables: Tables, grid, out: Optional[DecisionTable] = None, 
         out = alloc_decision_host(tables.n_tables, g.n_P, g.n_m)
     _check(lib.plogp_select_best_host(tables.handle, g.ref, out.strategy.data_ptr(), out.s_bytes.data_ptr(),
                                       out.time.data_ptr(), _stream_ptr(stream)), "plogp_select_best_host")
+    return out
+
+
+def n_candidates(grid) -> int:
+    """Number of candidate segment sizes of a grid (the last dimension of the surface)."""
+    g = _as_grid(grid)
+    if g.s is not None:
+        return len(g.s)
+    st = g.struct
+    return 0 if st.s_step == 0 or st.s_hi < st.s_lo else int((st.s_hi - st.s_lo) // st.s_step) + 1
+
+
+def segment_surface(tables: Tables, grid, out=None, stream=None):
+    """``plogp_segment_surface``: models of ids 2, 5, 9 for every candidate s, [n_tables][3][n_P][n_m][n_s]."""
+    import torch
+    g = _as_grid(grid)
+    if out is None:
+        out = torch.full((tables.n_tables, 3, g.n_P, g.n_m, n_candidates(g)), float("inf"), dtype=torch.float64, device="cuda")
+    _check(lib.plogp_segment_surface(tables.handle, g.ref, out.data_ptr(), _stream_ptr(stream)), "plogp_segment_surface")
+    return out
+
+
+def segment_sensitivity(tables: Tables, grid, s_fixed: int, pred: Optional[Prediction] = None, stream=None):
+    """``plogp_segment_sensitivity``: (time with the fixed segment size, its ratio to the searched minimum), each
+    [n_tables][3][n_P][n_m]; the ratio is None when no prediction is given."""
+    import torch
+    g = _as_grid(grid)
+    shape = (tables.n_tables, 3, g.n_P, g.n_m)
+    fixed = torch.full(shape, float("nan"), dtype=torch.float64, device="cuda")
+    ratio = None if pred is None else torch.full(shape, float("nan"), dtype=torch.float64, device="cuda")
+    _check(lib.plogp_segment_sensitivity(tables.handle, g.ref, int(s_fixed), None if pred is None else pred.time.data_ptr(),
+                                         fixed.data_ptr(), None if ratio is None else ratio.data_ptr(), _stream_ptr(stream)),
+           "plogp_segment_sensitivity")
+    return fixed, ratio
+
+
+def decision_boundaries(dec: DecisionTable, stream=None):
+    """``plogp_decision_boundaries``: uint8 flags [n_tables][2][n_P][n_m] (bit 0: changes with P, bit 1: with m)."""
+    import torch
+    n_tables, _, n_P, n_m = dec.strategy.shape
+    out = torch.empty_like(dec.strategy)
+    _check(lib.plogp_decision_boundaries(n_tables, n_P, n_m, dec.strategy.data_ptr(), out.data_ptr(), _stream_ptr(stream)),
+           "plogp_decision_boundaries")
     return out
