@@ -309,7 +309,7 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
         pl.n_pairs = n_m;
         pl.off_pair_base = append_aligned(blob, pair_base);
         // short lists: small CTAs; the list of representatives of one message size lives in shared memory
-        pl.env_threads = ns_max <= 64 ? 64 : 256;
+        pl.env_threads = ns_max <= 64 ? 64 : (ns_max <= 4096 ? 256 : 1024);
         pl.env_rep_cap = std::min(std::max(ns_max, 1), 6144);
         pl.env_coarse = std::max(64, (n_P + 1023) / 1024);
         pl.env_max_coarse = (std::max(n_P, 1) - 1 + pl.env_coarse - 1) / pl.env_coarse + 1;

@@ -30,18 +30,18 @@ constexpr unsigned kFull = 0xffffffffu;
 
 }  // namespace
 
-__global__ void __launch_bounds__(256) envelope_kernel(const EnvParams p)
+__global__ void __launch_bounds__(1024) envelope_kernel(const EnvParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int npad = p.T.npad, T = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = T >> 5;
     double *s_tab = reinterpret_cast<double *>(smem_raw);
     double *s_B = s_tab + 3 * npad;                                   // [rep_cap]
     double *s_C = s_B + p.rep_cap;                                    // [rep_cap]
-    double *s_redt = s_C + p.rep_cap;                                 // [8]
-    uint32_t *s_I = reinterpret_cast<uint32_t *>(s_redt + 8);         // [rep_cap] candidate index of an entry
+    double *s_redt = s_C + p.rep_cap;                                 // [32]
+    uint32_t *s_I = reinterpret_cast<uint32_t *>(s_redt + 32);        // [rep_cap] candidate index of an entry
     uint32_t *s_k = s_I + p.rep_cap;                                  // [T] exchange of k
     int *s_opt = reinterpret_cast<int *>(s_k + T);                    // [max_coarse]
-    int *s_cnt = s_opt + p.max_coarse;                                // [8] + [8]
+    int *s_cnt = s_opt + p.max_coarse;                                // [32] + [32]
 
     const int midx = blockIdx.x, trel = blockIdx.y, table = p.table0 + trel;
     const uint32_t m_u = p.G.m_list[midx];
@@ -61,32 +61,47 @@ __global__ void __launch_bounds__(256) envelope_kernel(const EnvParams p)
     double qmin = CUDART_INF;
     int qidx = 0x7FFFFFFF;
     int n_rep = 0;  // all representatives (of every window), known after the first pass
+    constexpr int V = 4;  // consecutive candidates per thread and chunk (independent searches and divisions in flight)
     auto list_pass = [&](int win) {
         int base = 0;
         uint32_t carry_k = 0;  // thread 0: k of the last candidate of the previous chunk
-        for (int c0 = 0; c0 < ns; c0 += T) {
-            const int si = c0 + tid;
-            const bool valid = si < ns;
-            double gs = 0.0;
-            uint32_t k = 0;
-            if (valid) {
-                const uint32_t s = s_at(p.G, si);
-                gs = gap_at(s_tab, npad, static_cast<double>(s));
-                k = segments(m_u, s, p.G.k_mode);
-                if (win == 0) {
-                    const double Q = gs * static_cast<double>(k);
-                    if (Q < qmin) { qmin = Q; qidx = si; }  // ascending si per thread: the smallest index stays
+        for (int c0 = 0; c0 < ns; c0 += V * T) {
+            double gs[V];
+            uint32_t k[V];
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                const int si = c0 + V * tid + v;
+                gs[v] = 0.0;
+                k[v] = 0;
+                if (si < ns) {
+                    const uint32_t s = s_at(p.G, si);
+                    gs[v] = gap_at(s_tab, npad, static_cast<double>(s));
+                    k[v] = segments(m_u, s, p.G.k_mode);
+                    if (win == 0) {
+                        const double Q = gs[v] * static_cast<double>(k[v]);
+                        if (Q < qmin) { qmin = Q; qidx = si; }  // ascending si per thread: the smallest index stays
+                    }
                 }
             }
-            s_k[tid] = k;
+            s_k[tid] = k[V - 1];
             __syncthreads();
-            bool rep = false;
-            if (valid) {
-                const uint32_t k_prev = tid > 0 ? s_k[tid - 1] : carry_k;
-                rep = si == 0 || k != k_prev;
+            uint32_t k_prev = tid > 0 ? s_k[tid - 1] : carry_k;
+            unsigned rep = 0;  // bit v: candidate v starts a run of equal segment count
+            int cnt = 0;
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                const int si = c0 + V * tid + v;
+                if (si < ns && (si == 0 || k[v] != k_prev)) { rep |= 1u << v; ++cnt; }
+                k_prev = k[v];
             }
-            const unsigned bal = __ballot_sync(kFull, rep);
-            if (lane == 0) s_cnt[warp] = __popc(bal);
+            // ordered positions: inclusive scan of the counts over the warp, then the warps' totals
+            int incl = cnt;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int y = __shfl_up_sync(kFull, incl, off);
+                if (lane >= off) incl += y;
+            }
+            if (lane == 31) s_cnt[warp] = incl;
             if (tid == 0) carry_k = s_k[T - 1];
             __syncthreads();
             int off = 0, total = 0;
@@ -95,12 +110,16 @@ __global__ void __launch_bounds__(256) envelope_kernel(const EnvParams p)
                 off += w < warp ? c : 0;
                 total += c;
             }
-            if (rep) {
-                const int pos = base + off + __popc(bal & ((1u << lane) - 1u)) - win * p.rep_cap;
-                if (pos >= 0 && pos < p.rep_cap) {
-                    s_B[pos] = gs + L;
-                    s_C[pos] = gs * (static_cast<double>(k) - 1.0);
-                    s_I[pos] = static_cast<uint32_t>(si);
+            int pos = base + off + incl - cnt - win * p.rep_cap;
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                if ((rep >> v) & 1u) {
+                    if (pos >= 0 && pos < p.rep_cap) {
+                        s_B[pos] = gs[v] + L;
+                        s_C[pos] = gs[v] * (static_cast<double>(k[v]) - 1.0);
+                        s_I[pos] = static_cast<uint32_t>(c0 + V * tid + v);
+                    }
+                    ++pos;
                 }
             }
             base += total;
@@ -112,13 +131,13 @@ __global__ void __launch_bounds__(256) envelope_kernel(const EnvParams p)
     // ---- ids 2 and 9: the smallest Q (smallest s on ties) serves every process count ----
     if (has2 || has9) {
         warp_min_pair(qmin, qidx);
-        if (lane == 0) { s_redt[warp] = qmin; s_cnt[8 + warp] = qidx; }
+        if (lane == 0) { s_redt[warp] = qmin; s_cnt[32 + warp] = qidx; }
         __syncthreads();
         double q = s_redt[0];
-        int qi = s_cnt[8];
+        int qi = s_cnt[32];
         for (int w = 1; w < n_warps; ++w) {
             const double q2 = s_redt[w];
-            const int i2 = s_cnt[8 + w];
+            const int i2 = s_cnt[32 + w];
             if (q2 < q || (q2 == q && i2 < qi)) { q = q2; qi = i2; }
         }
         for (int pidx = tid; pidx < n_P; pidx += T) {
@@ -182,8 +201,8 @@ __global__ void __launch_bounds__(256) envelope_kernel(const EnvParams p)
 
 size_t envelope_smem_bytes(const TableDev &T, int threads, int rep_cap, int max_coarse)
 {
-    return (3 * static_cast<size_t>(T.npad) + 2 * static_cast<size_t>(rep_cap) + 8) * sizeof(double) +
-           (static_cast<size_t>(rep_cap) + threads) * sizeof(uint32_t) + (static_cast<size_t>(max_coarse) + 16) * sizeof(int);
+    return (3 * static_cast<size_t>(T.npad) + 2 * static_cast<size_t>(rep_cap) + 32) * sizeof(double) +
+           (static_cast<size_t>(rep_cap) + threads) * sizeof(uint32_t) + (static_cast<size_t>(max_coarse) + 64) * sizeof(int);
 }
 
 cudaError_t launch_envelope(const EnvParams &p, int threads, cudaStream_t st)
