@@ -96,6 +96,25 @@ double po_model(const po_table *t, int strategy, int64_t P, uint64_t m, uint64_t
         for (int j = 0; j < d; ++j) acc += (long double)po_gap(t, ((uint64_t)1 << j) * m);
         return (double)acc + lc * L;
     }
+    /* ---- derived collectives (see the header): mirrored strategies, and a Barrier of one-byte messages ---- */
+    case 13: return po_model(t, 10, P, m, s, k_mode); /* Gather Flat Tree */
+    case 14: return po_model(t, 11, P, m, s, k_mode); /* Gather Chain */
+    case 15: return po_model(t, 12, P, m, s, k_mode); /* Gather Binomial Tree */
+    case 16: return po_model(t, 0, P, m, s, k_mode);  /* Reduce Flat Tree */
+    case 17: return po_model(t, 2, P, m, s, k_mode);  /* Reduce Segmented Flat Tree */
+    case 18: return po_model(t, 3, P, m, s, k_mode);  /* Reduce Chain */
+    case 19: return po_model(t, 5, P, m, s, k_mode);  /* Reduce Segmented Chain */
+    case 20: return po_model(t, 6, P, m, s, k_mode);  /* Reduce Binary Tree */
+    case 21: return po_model(t, 7, P, m, s, k_mode);  /* Reduce Binomial Tree */
+    case 22: return po_model(t, 9, P, m, s, k_mode);  /* Reduce Segmented Binomial Tree */
+    case 23: /* Barrier Flat Tree: 2 ((P-1) g(1) + L) */
+        return 2.0 * (Pm1 * po_gap(t, 1) + L);
+    case 24: /* Barrier Chain: 2 (P-1) (g(1) + L) */
+        return 2.0 * (Pm1 * (po_gap(t, 1) + L));
+    case 25: /* Barrier Binary Tree: 2 ceil(log2 P) (2 g(1) + L) */
+        return 2.0 * (lc * (2.0 * po_gap(t, 1) + L));
+    case 26: /* Barrier Binomial Tree: 2 (floor(log2 P) g(1) + ceil(log2 P) L) */
+        return 2.0 * (lf * po_gap(t, 1) + lc * L);
     default:
         return NAN;
     }
@@ -144,14 +163,16 @@ void po_segment_search(const po_table *t, int strategy, int64_t P, uint64_t m, c
     *runner_up = ru;
 }
 
-static int is_segmented(int id) { return id == 2 || id == 5 || id == 9; }
+static int is_segmented(int id) { return id == 2 || id == 5 || id == 9 || id == 17 || id == 19 || id == 22; }
 
 /* ---- Sections 1 and 5: pick the strategy with the lowest prediction ---- */
 int po_decide(const po_table *t, int collective, uint32_t mask, int64_t P, uint64_t m,
               const po_sgrid *sg, int k_mode, int *strategy_out, uint64_t *s_out, double *time_out,
               double *runner_up)
 {
-    int lo = collective == 0 ? 0 : 10, hi = collective == 0 ? 10 : 13;
+    static const int first[6] = {0, 10, 13, 16, 23, 27};
+    if (collective < 0 || collective > 4) return -1;
+    int lo = first[collective], hi = first[collective + 1];
     double bt = INFINITY, ru = INFINITY;
     int bid = -1;
     uint64_t bs = 0;
@@ -288,6 +309,24 @@ void po_fixed_segment_grid(const po_table *t, uint32_t mask, const int64_t *P, i
                 time_fixed[((size_t)q * n_P + ip) * n_m + im] =
                     po_model(t, seg_ids[q], P[ip], m[im], po_effective_segment(m[im], s_fixed), k_mode);
     }
+}
+
+void po_decide_grid(const po_table *t, int collective, uint32_t mask, const int64_t *P, int n_P, const uint64_t *m, int n_m,
+                    const po_sgrid *sg, int k_mode, uint8_t *strategy, uint64_t *s_out, double *time_out, double *runner_up)
+{
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int ip = 0; ip < n_P; ++ip)
+        for (int im = 0; im < n_m; ++im) {
+            size_t cell = (size_t)ip * n_m + im;
+            int id = 255;
+            uint64_t s = 0;
+            double v = NAN, ru = NAN;
+            if (po_decide(t, collective, mask, P[ip], m[im], sg, k_mode, &id, &s, &v, &ru) != 0) id = 255;
+            strategy[cell] = (uint8_t)id;
+            s_out[cell] = s;
+            time_out[cell] = v;
+            runner_up[cell] = ru;
+        }
 }
 
 int po_threads(void)

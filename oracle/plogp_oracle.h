@@ -33,6 +33,25 @@
  *   2 Segmented Flat Tree       7 Binomial Tree                12 Scatter Binomial Tree
  *   3 Chain                     8 Binomial Tree Rendezvous
  *   4 Chain Rendezvous          9 Segmented Binomial Tree
+ *
+ * Collectives the paper names but prints no models for (Section 3: Barrier, Reduce and Gather are built "in a very
+ * similar way" as Broadcast and Scatter).  Their models here are derived, not printed: with the gap charged to a
+ * node's port for receives as for sends (in Table 1 / Table 2 no node ever receives two messages at once, so the
+ * paper never needs that rule), a Gather is a Scatter run backwards in time and a Reduce a Broadcast run backwards
+ * (communication only: pLogP has no parameter for the combine operation), so their times are those of the mirrored
+ * strategy; a Barrier is a Reduce followed by a Broadcast of one-byte messages, g(1) being the gap the paper's
+ * rendezvous rows already use for an empty message.  "parity unpinned" by the paper; pinned here by the
+ * send-schedule simulation with a receive port.
+ *  13 Gather Flat Tree          (P-1) g(m) + L                                   (= id 10)
+ *  14 Gather Chain              sum_{j=1..P-1} g(j m) + (P-1) L                  (= id 11)
+ *  15 Gather Binomial Tree      sum_{j=0..ceil(log2 P)-1} g(2^j m) + ceil(log2 P) L   (= id 12)
+ *  16 Reduce Flat Tree (= 0)    17 Reduce Segmented Flat Tree (= 2)   18 Reduce Chain (= 3)
+ *  19 Reduce Segmented Chain (= 5)   20 Reduce Binary Tree (= 6)   21 Reduce Binomial Tree (= 7)
+ *  22 Reduce Segmented Binomial Tree (= 9)
+ *  23 Barrier Flat Tree         2 ((P-1) g(1) + L)
+ *  24 Barrier Chain             2 (P-1) (g(1) + L)
+ *  25 Barrier Binary Tree       2 ceil(log2 P) (2 g(1) + L)
+ *  26 Barrier Binomial Tree     2 (floor(log2 P) g(1) + ceil(log2 P) L)
  */
 #ifndef PLOGP_ORACLE_H
 #define PLOGP_ORACLE_H
@@ -82,7 +101,8 @@ void po_segment_search(const po_table *t, int strategy, int64_t P, uint64_t m, c
                        int k_mode, uint64_t *best_s, double *best_time, double *runner_up);
 
 /* Strategy selection for one (collective, P, m): collective 0 = Broadcast
- * (ids 0..9), 1 = Scatter (ids 10..12); only ids enabled in mask compete.
+ * (ids 0..9), 1 = Scatter (ids 10..12), 2 = Gather (13..15), 3 = Reduce (16..22), 4 = Barrier (23..26, m is
+ * ignored); only ids enabled in mask (bit i = id i) compete.
  * s_out = 0 when the winner is unsegmented.  runner_up = best time of the
  * best OTHER strategy (+inf if none).  Returns 0, or -1 when no strategy of
  * that collective is enabled (outputs untouched). */
@@ -121,6 +141,12 @@ void po_surface_grid(const po_table *t, uint32_t mask, const int64_t *P, int n_P
 /* time_fixed[q][ip][im] = po_model(id_q, P, m, po_effective_segment(m, s_fixed)); disabled ids untouched. */
 void po_fixed_segment_grid(const po_table *t, uint32_t mask, const int64_t *P, int n_P, const uint64_t *m,
                            int n_m, uint64_t s_fixed, int k_mode, double *time_fixed);
+
+/* po_decide over a grid (OpenMP over cells): strategy / s / time / runner_up, each [n_P][n_m]. */
+void po_decide_grid(const po_table *t, int collective, uint32_t mask, const int64_t *P, int n_P, const uint64_t *m, int n_m,
+                    const po_sgrid *sg, int k_mode, uint8_t *strategy, uint64_t *s_out, double *time_out, double *runner_up);
+
+#define PO_N_MODELS 27
 
 int po_threads(void);
 

@@ -89,6 +89,9 @@ def _load():
         lib.po_fixed_segment_grid.restype = None
         lib.po_fixed_segment_grid.argtypes = [TP, C.c_uint32, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_uint64,
                                               C.c_int, C.c_void_p]
+        lib.po_decide_grid.restype = None
+        lib.po_decide_grid.argtypes = [TP, C.c_int, C.c_uint32, C.c_void_p, C.c_int, C.c_void_p, C.c_int, SP, C.c_int,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.po_threads.restype = C.c_int
         _lib = lib
     return _lib
@@ -246,3 +249,24 @@ def decision_boundaries(strategy: np.ndarray) -> np.ndarray:
     out[..., :-1, :] |= (s[..., :-1, :] != s[..., 1:, :]).astype(np.uint8)
     out[..., :, :-1] |= ((s[..., :, :-1] != s[..., :, 1:]).astype(np.uint8) << 1)
     return out
+
+
+# Collectives the paper names without printing models (derived in plogp_oracle.h): ids and what they mirror
+GATHER, REDUCE, BARRIER = 2, 3, 4
+DERIVED_FIRST_ID = {GATHER: 13, REDUCE: 16, BARRIER: 23}
+MIRROR_OF = {13: 10, 14: 11, 15: 12, 16: 0, 17: 2, 18: 3, 19: 5, 20: 6, 21: 7, 22: 9}   # derived id -> printed id
+BARRIER_SHAPE_OF = {23: 0, 24: 3, 25: 6, 26: 7}                                           # barrier id -> tree shape's Broadcast id
+
+
+def decide_grid(t: Table, collective: int, mask: int, P, m, sg: SGrid, k_mode: int = 0) -> Decision:
+    """po_decide for every (P, m): Decision with [n_P][n_m] arrays (strategy 255 where nothing is enabled)."""
+    P = np.ascontiguousarray(P, dtype=np.int64)
+    m = np.ascontiguousarray(m, dtype=np.uint64)
+    nP, nm = len(P), len(m)
+    strategy = np.zeros((nP, nm), dtype=np.uint8)
+    s = np.zeros((nP, nm), dtype=np.uint64)
+    time = np.zeros((nP, nm), dtype=np.float64)
+    ru = np.zeros((nP, nm), dtype=np.float64)
+    _load().po_decide_grid(t.ref, int(collective), int(mask), P.ctypes.data, nP, m.ctypes.data, nm, sg.ref, int(k_mode),
+                           strategy.ctypes.data, s.ctypes.data, time.ctypes.data, ru.ctypes.data)
+    return Decision(strategy, s, time, ru)

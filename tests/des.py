@@ -4,8 +4,14 @@ pLogP semantics used (Section 2 of the paper; the same ones that make Table 1's
 Flat Tree equal (P-1) g(m) + L and its Chain equal (P-1)(g(m) + L)): a node has
 one send port, busy for g(size) per message it sends; a message whose
 transmission starts at time t is available at its receiver at t + g(size) + L;
-receiving is free; a node issues its sends in program order, each as soon as
-the port is free and the data it depends on has arrived.
+a node issues its sends in program order, each as soon as the port is free and
+the data it depends on has arrived.  Receiving costs the receiver's port the
+same gap: reception starts L after the send started, or when the receiver has
+finished its previous reception if that is later, and lasts g(size).  In the
+paper's Broadcast and Scatter strategies no node ever receives two messages at
+once, so this rule never shows there (arrival = t + g(size) + L); it is what
+makes a Gather or a Reduce — many senders, one receiver — take the mirrored
+strategy's time.
 
 Nothing here uses the closed-form models: a schedule is a list of sends with
 dependencies, and the completion time is the latest arrival.
@@ -31,6 +37,7 @@ def simulate(n_nodes: int, sends: List[Send], g: Callable[[int], float], L: floa
         queues[s.src].append(i)
     heads = [0] * n_nodes
     port_free = [0.0] * n_nodes
+    rx_free = [0.0] * n_nodes
     arrival: List[Optional[float]] = [None] * len(sends)
     remaining = len(sends)
     while remaining:
@@ -49,7 +56,9 @@ def simulate(n_nodes: int, sends: List[Send], g: Callable[[int], float], L: floa
         start, node, i = best
         busy = g(sends[i].size)
         port_free[node] = start + busy
-        arrival[i] = start + busy + L
+        dst = sends[i].dst
+        arrival[i] = max(start + L, rx_free[dst]) + busy
+        rx_free[dst] = arrival[i]
         heads[node] += 1
         remaining -= 1
     return max(arrival) if sends else 0.0
@@ -175,3 +184,98 @@ def scatter_chain(P: int, m: int) -> List[Send]:
 def scatter_binomial(P: int, m: int) -> List[Send]:
     """A child receives its own block and those of its whole subtree."""
     return _tree_schedule(_binomial_edges(P), lambda n: n * m)
+
+
+# ---------------- the mirrored collectives: many senders, one receiver ----------------
+
+def _reversed_tree(edges, size_of: Callable[[int], int], k: int = 1) -> List[Send]:
+    """Every edge (parent, child, subtree size) carries k messages from the child to the parent; a child sends
+    only after all messages of all its own children have arrived (the mirror image of _tree_schedule)."""
+    children = {}
+    for (p, c, n) in edges:
+        children.setdefault(p, []).append((c, n))
+    out: List[Send] = []
+
+    def emit(node: int) -> List[int]:
+        """Schedules the subtree below node; returns the ids of the sends that arrive at node."""
+        incoming: List[int] = []
+        for (c, n) in reversed(children.get(node, [])):   # smallest subtree first: the reverse of the send order
+            below = emit(c)
+            for _ in range(k):
+                incoming.append(len(out))
+                out.append(Send(c, node, size_of(n), tuple(below)))
+        return incoming
+
+    emit(0)
+    return out
+
+
+def _flat_edges(P: int):
+    return [(0, d, 1) for d in range(1, P)]
+
+
+def gather_flat(P: int, m: int) -> List[Send]:
+    return _reversed_tree(_flat_edges(P), lambda n: m)
+
+
+def gather_chain(P: int, m: int) -> List[Send]:
+    """Node i passes on its own block and those of everybody behind it: (P-i) blocks of m."""
+    out: List[Send] = []
+    for i in range(P - 1, 0, -1):
+        out.append(Send(i, i - 1, (P - i) * m, (len(out) - 1,) if i < P - 1 else ()))
+    return out
+
+
+def gather_binomial(P: int, m: int) -> List[Send]:
+    return _reversed_tree(_binomial_edges(P), lambda n: n * m)
+
+
+def reduce_flat(P: int, m: int) -> List[Send]:
+    return _reversed_tree(_flat_edges(P), lambda n: m)
+
+
+def reduce_segmented_flat(P: int, s: int, k: int) -> List[Send]:
+    return _reversed_tree(_flat_edges(P), lambda n: s, k)
+
+
+def reduce_chain(P: int, m: int) -> List[Send]:
+    out: List[Send] = []
+    for i in range(P - 1, 0, -1):
+        out.append(Send(i, i - 1, m, (len(out) - 1,) if i < P - 1 else ()))
+    return out
+
+
+def reduce_segmented_chain(P: int, s: int, k: int) -> List[Send]:
+    """Each node passes a segment on as soon as that segment has arrived from behind."""
+    out: List[Send] = []
+    idx = {}
+    for i in range(P - 1, 0, -1):
+        for c in range(k):
+            idx[(i, c)] = len(out)
+            out.append(Send(i, i - 1, s, (idx[(i + 1, c)],) if i < P - 1 else ()))
+    return out
+
+
+def reduce_binomial(P: int, m: int) -> List[Send]:
+    return _reversed_tree(_binomial_edges(P), lambda n: m)
+
+
+def reduce_segmented_binomial(P: int, s: int, k: int) -> List[Send]:
+    return _reversed_tree(_binomial_edges(P), lambda n: s, k)
+
+
+def _binary_edges(P: int):
+    return [(node, child, 1) for node in range(P) for child in (2 * node + 1, 2 * node + 2) if child < P]
+
+
+def reduce_binary(P: int, m: int) -> List[Send]:
+    return _reversed_tree(_binary_edges(P), lambda n: m)
+
+
+def barrier(P: int, up: List[Send], down: List[Send]) -> List[Send]:
+    """A reduction of one-byte messages (up) followed by a broadcast of one-byte messages (down): the root's first
+    broadcast sends wait for everything that arrives at the root."""
+    last = tuple(i for i, snd in enumerate(up) if snd.dst == 0)
+    off = len(up)
+    shifted = [Send(snd.src, snd.dst, snd.size, tuple(d + off for d in snd.needs) + (last if snd.src == 0 else ())) for snd in down]
+    return list(up) + shifted
