@@ -149,6 +149,29 @@ int plogp_select_best(plogp_tables *tables, const plogp_grid *grid, uint8_t *d_s
                       uint32_t *d_s_bytes, double *d_time, void *stream);
 
 /*
+ * Decision tables for the collectives that Section 3 names as built "in a very similar way" as Broadcast and Scatter
+ * — Gather, Reduce, Barrier — but for which the paper prints no models.  The models used here are derived (the
+ * paper has no counterpart to cite for the formulas themselves): with the gap charged to a node's port for receives
+ * as for sends, a Gather is a Scatter run backwards in time and a Reduce a Broadcast run backwards (communication
+ * only: pLogP has no parameter for the combine operation), so each takes the mirrored strategy's time; a Barrier is a
+ * Reduce followed by a Broadcast of one-byte messages.
+ *   collective   PLOGP_GATHER:  ids 13 Flat Tree, 14 Chain, 15 Binomial Tree              (mirrors of ids 10, 11, 12)
+ *                PLOGP_REDUCE:  ids 16 Flat, 17 Segmented Flat, 18 Chain, 19 Segmented Chain, 20 Binary, 21 Binomial,
+ *                               22 Segmented Binomial Tree                                (mirrors of ids 0 2 3 5 6 7 9)
+ *                PLOGP_BARRIER: ids 23 Flat Tree 2((P-1) g(1) + L), 24 Chain 2 (P-1)(g(1) + L),
+ *                               25 Binary Tree 2 ceil(log2 P)(2 g(1) + L), 26 Binomial Tree 2 (floor(log2 P) g(1) + ceil(log2 P) L)
+ *   grid->strategy_mask  bit i enables the strategy that mirrors printed id i (Barrier: the tree shape of ids 0, 3, 6, 7);
+ *                other bits are ignored.  All other grid fields as in plogp_select_best.
+ *   d_strategy / d_s_bytes / d_time   DEVICE, one plane per table: [n_tables][n_P][n_m]; for PLOGP_BARRIER
+ *                [n_tables][n_P] (the message sizes play no part, but the grid must still carry at least one).
+ * A collective with no enabled strategy leaves its outputs untouched.  Same stream and ownership rules as
+ * plogp_select_best; Gather and Reduce run the same kernels.
+ */
+enum { PLOGP_GATHER = 2, PLOGP_REDUCE = 3, PLOGP_BARRIER = 4 };
+int plogp_select_best_collective(plogp_tables *tables, const plogp_grid *grid, int collective, uint8_t *d_strategy,
+                                 uint32_t *d_s_bytes, double *d_time, void *stream);
+
+/*
  * plogp_select_best with HOST outputs: the same decision table (Sections 1 and 5), delivered into the
  * caller's host arrays h_strategy / h_s_bytes / h_time, each [n_tables][2][n_P][n_m].  The tables are
  * processed in batches through two device staging sets owned by the handle (at most 512 MiB each, or one

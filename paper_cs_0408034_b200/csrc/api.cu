@@ -387,6 +387,15 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// plogp_select_best's layout: two planes per table, the ids of Table 1 / Table 2
+OutMap default_out_map()
+{
+    OutMap om{};
+    om.planes = 2; om.plane_bcast = 0; om.plane_scat = 1;
+    for (int i = 0; i < 16; ++i) om.id_of[i] = uint8_t(i < PLOGP_N_STRATEGIES ? i : 255);
+    return om;
+}
+
 int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cudaStream_t st, int t_begin = 0, int t_end = -1)
 {
     int dev = 0;
@@ -456,7 +465,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             dp.T = h->T; dp.G = pl.G;
             dp.G.mask &= 0x3FFu;
             dp.n_mgroups = pl.dec_mgroups; dp.n_ptiles = pl.dec_ptiles; dp.mg = pl.dec_mg;
-            dp.table0 = t0; dp.n_tables_launch = nt; dp.out_table0 = out.out_table0;
+            dp.table0 = t0; dp.n_tables_launch = nt; dp.out_table0 = out.out_table0; dp.om = out.om;
             dp.d_strategy = out.d_strategy; dp.d_sbytes = out.d_sbytes; dp.d_time = out.d_time;
             dp.envelope = pl.envelope_short ? 1 : 0;
             dp.vec_out = (pl.G.n_m % 2 == 0) && pl.dec_mg >= 2 && reinterpret_cast<uintptr_t>(out.d_time) % 16 == 0 &&
@@ -637,6 +646,7 @@ int plogp_predict(plogp_tables *tables, const plogp_grid *grid, double *d_time, 
 {
     if (!tables || !grid || !d_time) return PLOGP_E_INVAL;
     FusedParams out{};
+    out.om = default_out_map();
     out.p_time = d_time;
     out.p_best_s = d_best_s;
     return run(tables, grid, true, out, static_cast<cudaStream_t>(stream));
@@ -647,6 +657,7 @@ int plogp_select_best(plogp_tables *tables, const plogp_grid *grid, uint8_t *d_s
 {
     if (!tables || !grid || !d_strategy || !d_s_bytes || !d_time) return PLOGP_E_INVAL;
     FusedParams out{};
+    out.om = default_out_map();
     out.d_strategy = d_strategy;
     out.d_sbytes = d_s_bytes;
     out.d_time = d_time;
@@ -702,6 +713,7 @@ int plogp_select_best_host(plogp_tables *h, const plogp_grid *grid, uint8_t *h_s
             if (ew != cudaSuccess) { rc = cuda_fail(ew, "cudaStreamWaitEvent"); break; }
         }
         FusedParams out{};
+        out.om = default_out_map();
         out.d_time = s_time;
         out.d_sbytes = s_sb;
         out.d_strategy = s_id;
@@ -727,6 +739,44 @@ int plogp_select_best_host(plogp_tables *h, const plogp_grid *grid, uint8_t *h_s
     if (e1 != cudaSuccess) return cuda_fail(e1, "cudaStreamSynchronize(copy)");
     if (e2 != cudaSuccess) return cuda_fail(e2, "cudaStreamSynchronize");
     return PLOGP_OK;
+}
+
+int plogp_select_best_collective(plogp_tables *h, const plogp_grid *grid, int collective, uint8_t *d_strategy,
+                                 uint32_t *d_s_bytes, double *d_time, void *stream)
+{
+    if (!h || !grid || !d_strategy || !d_s_bytes || !d_time) return PLOGP_E_INVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    plogp_grid g = *grid;
+    FusedParams out{};
+    out.om = default_out_map();
+    out.om.planes = 1; out.om.plane_bcast = 0; out.om.plane_scat = 0;
+    out.d_strategy = d_strategy; out.d_sbytes = d_s_bytes; out.d_time = d_time;
+    switch (collective) {
+    case PLOGP_GATHER:  // the Scatter strategies run backwards: ids 10, 11, 12 -> 13, 14, 15
+        g.strategy_mask &= 0x1C00u;
+        for (int i = 10; i <= 12; ++i) out.om.id_of[i] = uint8_t(i + 3);
+        return run(h, &g, false, out, st);
+    case PLOGP_REDUCE: {  // the Broadcast strategies without a handshake run backwards: 0 2 3 5 6 7 9 -> 16 .. 22
+        g.strategy_mask &= 0x2EDu;
+        static const int from[7] = {0, 2, 3, 5, 6, 7, 9};
+        for (int i = 0; i < 7; ++i) out.om.id_of[from[i]] = uint8_t(16 + i);
+        return run(h, &g, false, out, st);
+    }
+    case PLOGP_BARRIER: {  // one decision per (table, P); the message sizes play no part
+        g.strategy_mask &= 0xC9u;
+        int dev = 0;
+        CK(cudaGetDevice(&dev));
+        if (dev != h->device) return PLOGP_E_INVAL;
+        int rc = prepare(h, &g, st);
+        if (rc != PLOGP_OK) { h->plan = Plan(); return rc; }
+        if (h->plan.empty) return PLOGP_OK;  // no process count, no message size to carry the plan, or no strategy
+        CK(launch_barrier(h->T, h->plan.G, 0, h->T.n_tables, d_strategy, d_s_bytes, d_time, st));
+        g_launches += 1;
+        return PLOGP_OK;
+    }
+    default:
+        return PLOGP_E_INVAL;
+    }
 }
 
 int plogp_segment_surface(plogp_tables *h, const plogp_grid *grid, double *d_surface, void *stream)

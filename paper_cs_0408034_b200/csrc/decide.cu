@@ -390,7 +390,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
         if (mi < n_mi) {
             const uint32_t m_u0 = p.G.m_list[m0 + mi], m_u1 = p.G.m_list[m0 + mi + 1];
             const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
-            const size_t base = static_cast<size_t>(table - p.out_table0) * 2 * plane + static_cast<size_t>(m0 + mi);
+            const size_t base = (static_cast<size_t>(table - p.out_table0) * p.om.planes + p.om.plane_bcast) * plane + static_cast<size_t>(m0 + mi);
             const double *st0 = sm.st_time + mi * kStageStride, *st1 = st0 + kStageStride;
             const uint16_t *sc0 = sm.st_code + mi * kCodeStride, *sc1 = sc0 + kCodeStride;
             for (int pr = warp * rows + prow; pr < n_valid; pr += kDecWarps * rows) {
@@ -401,7 +401,8 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 const uint32_t s1 = cand1 == kCandNone ? 0u : (cand1 == kCandWhole ? m_u1 : sm.sval[cand1]);
                 *reinterpret_cast<double2 *>(p.d_time + o) = make_double2(st0[pr], st1[pr]);
                 *reinterpret_cast<uint2 *>(p.d_sbytes + o) = make_uint2(s0, s1);
-                *reinterpret_cast<uint16_t *>(p.d_strategy + o) = static_cast<uint16_t>((code0 >> 8) | (code1 & 0xFF00u));
+                *reinterpret_cast<uint16_t *>(p.d_strategy + o) =
+                    static_cast<uint16_t>(p.om.id_of[(code0 >> 8) & 15u] | (static_cast<uint32_t>(p.om.id_of[(code1 >> 8) & 15u]) << 8));
             }
         }
     } else {
@@ -409,13 +410,13 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
         if (mi < n_mi) {
             const uint32_t m_u = p.G.m_list[m0 + mi];
             const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
-            const size_t base = static_cast<size_t>(table - p.out_table0) * 2 * plane + static_cast<size_t>(m0 + mi);
+            const size_t base = (static_cast<size_t>(table - p.out_table0) * p.om.planes + p.om.plane_bcast) * plane + static_cast<size_t>(m0 + mi);
             for (int pr = warp * rows + prow; pr < n_valid; pr += kDecWarps * rows) {
                 const size_t o = base + static_cast<size_t>(tile0 + pr) * p.G.n_m;
                 const uint32_t code = sm.st_code[mi * kCodeStride + pr];
                 const uint32_t cand = code & 255u;
                 p.d_time[o] = sm.st_time[mi * kStageStride + pr];
-                p.d_strategy[o] = static_cast<uint8_t>(code >> 8);
+                p.d_strategy[o] = p.om.id_of[(code >> 8) & 15u];
                 p.d_sbytes[o] = cand == kCandNone ? 0u : (cand == kCandWhole ? m_u : sm.sval[cand]);
             }
         }

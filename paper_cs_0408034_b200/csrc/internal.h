@@ -13,6 +13,16 @@ namespace plogp {
 //   slope[npad] (g[i+1]-g[i]) / (size[i+1]-size[i])
 // npad is a power of two >= n_bp, so the interval search needs no bounds checks and an upward
 // walk always meets a +inf key.
+// Where a decision kernel puts its results and how it names the strategies.  plogp_select_best writes two planes
+// per table (Broadcast, Scatter) with the ids of Table 1 / Table 2; the derived collectives (Gather, Reduce) reuse
+// the same kernels with one plane per table and the ids of the mirrored strategies.
+struct OutMap {
+    int planes;       // decision planes per table in the output arrays
+    int plane_bcast;  // plane that receives the Broadcast-type decision
+    int plane_scat;   // plane that receives the Scatter-type decision
+    uint8_t id_of[16];  // output id of internal strategy id 0..12 (255 beyond)
+};
+
 struct TableDev {
     const double *tab;  // [n_tables][3*npad]
     const double *lat;  // [n_tables]
@@ -80,6 +90,7 @@ struct FusedParams {
     int n_mtiles, n_ptiles, passes_per_tile;  // a pass covers kWarps*R process counts
     int table0, n_tables_launch;
     int out_table0;  // table whose results sit at the start of the output arrays (0 unless the caller passes a window)
+    OutMap om;
     const double *s1_sums;  // [n_tables_launch][n_ptiles][9][n_m] Scatter Chain sums per warp run and per tile, or nullptr
     // segmented minima precomputed by the sweep kernel (nullptr => inline sweep)
     const double *part_time;
@@ -113,6 +124,7 @@ struct DecideParams {
     int vec_out;  // outputs aligned for two message sizes per store (n_m even, 16 / 8 / 2-byte aligned bases)
     int table0, n_tables_launch;
     int out_table0;  // table whose results sit at the start of the output arrays
+    OutMap om;
     uint8_t *d_strategy;
     uint32_t *d_sbytes;
     double *d_time;
@@ -141,6 +153,8 @@ cudaError_t launch_s1_tiles(const S1Params &p, cudaStream_t st);
 size_t decide_smem_bytes(const TableDev &T, const GridDev &G);
 cudaError_t launch_decide(const DecideParams &p, cudaStream_t st);
 cudaError_t launch_fp64_probe(double *d_sink, int iters, int blocks, cudaStream_t st);
+cudaError_t launch_barrier(const TableDev &T, const GridDev &G, int table0, int n_tables_launch, uint8_t *d_strategy, uint32_t *d_sbytes,
+                           double *d_time, cudaStream_t st);
 cudaError_t launch_surface(const SensParams &p, cudaStream_t st);
 cudaError_t launch_fixed(const SensParams &p, cudaStream_t st);
 cudaError_t launch_boundaries(const uint8_t *d_strategy, uint8_t *d_boundary, long long n_planes, int n_P, int n_m, int sm_count, cudaStream_t st);

@@ -412,8 +412,8 @@ __global__ void __launch_bounds__(kThreads, 2) fused_kernel(const FusedParams p)
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
                     if (ok[r] && m_ok) {
-                        const size_t o = out_index(coll, 2, r);
-                        p.d_strategy[o] = static_cast<uint8_t>(bid[r]);
+                        const size_t o = out_index(coll == 0 ? p.om.plane_bcast : p.om.plane_scat, p.om.planes, r);
+                        p.d_strategy[o] = bid[r] < 16 ? p.om.id_of[bid[r]] : static_cast<uint8_t>(bid[r]);
                         p.d_sbytes[o] = bsz[r];
                         p.d_time[o] = bt[r];
                     }

@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
     double x = static_cast<double>(P0 - 1) * md;
 
     const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
-    size_t o = (static_cast<size_t>(table - p.out_table0) * 2 + 1) * plane + static_cast<size_t>(e0) * p.G.n_m + midx;
+    size_t o = (static_cast<size_t>(table - p.out_table0) * p.om.planes + p.om.plane_scat) * plane + static_cast<size_t>(e0) * p.G.n_m + midx;
     int P = P0;
     int lc = 32 - __clz(P - 1);               // ceil(log2 P)
     int P_next_lc = (1 << lc) + 1;            // first process count with a larger ceil(log2 P)
@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
         }
         if (on12 && s2 < bt) { bt = s2; bid = 12; }                      // Binomial Tree
         p.d_time[o] = bt;
-        p.d_strategy[o] = static_cast<uint8_t>(bid);
+        p.d_strategy[o] = bid < 16 ? p.om.id_of[bid] : static_cast<uint8_t>(bid);
         p.d_sbytes[o] = 0u;
         o += p.G.n_m;
         if (CONTIG) { ++P; pm1 += 1.0; }

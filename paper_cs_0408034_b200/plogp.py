@@ -20,7 +20,8 @@ N_STRATEGIES = 13
 SEGMENTED_IDS = (2, 5, 9)
 EXPORTS = ("plogp_table_load", "plogp_table_update", "plogp_table_free", "plogp_predict", "plogp_select_best", "plogp_select_best_host",
            "plogp_status_string", "plogp_last_cuda_error", "plogp_kernel_launches", "plogp_fp64_fma_rate", "plogp_profile_enable", "plogp_profile_read",
-           "plogp_scatter_chain_static", "plogp_segment_surface", "plogp_segment_sensitivity", "plogp_decision_boundaries")
+           "plogp_scatter_chain_static", "plogp_segment_surface", "plogp_segment_sensitivity", "plogp_decision_boundaries",
+           "plogp_select_best_collective")
 
 OK, E_INVAL, E_NOMEM, E_CUDA, E_RANGE = 0, -1, -2, -3, -4
 
@@ -69,6 +70,8 @@ lib.plogp_segment_sensitivity.restype = C.c_int
 lib.plogp_segment_sensitivity.argtypes = [C.c_void_p, C.POINTER(Grid), C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.plogp_decision_boundaries.restype = C.c_int
 lib.plogp_decision_boundaries.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+lib.plogp_select_best_collective.restype = C.c_int
+lib.plogp_select_best_collective.argtypes = [C.c_void_p, C.POINTER(Grid), C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.plogp_profile_enable.restype = C.c_int
 lib.plogp_profile_enable.argtypes = [C.c_void_p, C.c_int]
 lib.plogp_profile_read.restype = C.c_int
@@ -353,4 +356,21 @@ def decision_boundaries(dec: DecisionTable, stream=None):
     out = torch.empty_like(dec.strategy)
     _check(lib.plogp_decision_boundaries(n_tables, n_P, n_m, dec.strategy.data_ptr(), out.data_ptr(), _stream_ptr(stream)),
            "plogp_decision_boundaries")
+    return out
+
+
+GATHER, REDUCE, BARRIER = 2, 3, 4
+
+
+def select_best_collective(tables: Tables, grid, collective: int, stream=None) -> DecisionTable:
+    """``plogp_select_best_collective``: decision table of a derived collective (GATHER, REDUCE: [n_tables][n_P][n_m];
+    BARRIER: [n_tables][n_P])."""
+    import torch
+    g = _as_grid(grid)
+    shape = (tables.n_tables, g.n_P) if collective == BARRIER else (tables.n_tables, g.n_P, g.n_m)
+    out = DecisionTable(torch.full(shape, 255, dtype=torch.uint8, device="cuda"),
+                        torch.zeros(shape, dtype=torch.int32, device="cuda"),
+                        torch.full(shape, float("nan"), dtype=torch.float64, device="cuda"))
+    _check(lib.plogp_select_best_collective(tables.handle, g.ref, int(collective), out.strategy.data_ptr(), out.s_bytes.data_ptr(),
+                                            out.time.data_ptr(), _stream_ptr(stream)), "plogp_select_best_collective")
     return out
