@@ -248,15 +248,22 @@ def run_reference(args, rank):
 
 def predict_counts(w, counts):
     """Work of plogp_predict on a workload: the same model cells, but every enabled plane is written out
-    (8 B per cell, plus 4 B per cell for the best segment size of each segmented strategy)."""
+    (8 B per cell, plus 4 B per cell for the best segment size of each segmented strategy).  Short candidate
+    lists: segmin_kernel evaluates the segmented cells and writes their planes, fused_kernel the rest."""
     n_on = bin(w.strategy_mask).count("1")
     n_seg = sum((w.strategy_mask >> b) & 1 for b in (2, 5, 9))
-    out_bytes = w.n_tables * w.n_P * w.n_m * (8 * n_on + 4 * n_seg)
+    cells_pm = w.n_tables * w.n_P * w.n_m
+    out_bytes = cells_pm * (8 * n_on + 4 * n_seg)
+    seg_bytes = cells_pm * 12 * n_seg
     slots = counts["fp64_slots"]
+    seg_slots = 2 * counts["segmented_cells"]
     c = dict(counts)
     if "sweep_kernel" in counts["per_kernel"]:
         sweep = counts["per_kernel"]["sweep_kernel"]
         c["per_kernel"] = {"sweep_kernel": sweep, "fused_kernel": {"fp64_slots": slots - sweep["fp64_slots"], "hbm_bytes": out_bytes}}
+    elif n_seg:
+        c["per_kernel"] = {"segmin_kernel": {"fp64_slots": seg_slots, "hbm_bytes": seg_bytes},
+                           "fused_kernel": {"fp64_slots": slots - seg_slots, "hbm_bytes": out_bytes - seg_bytes}}
     else:
         c["per_kernel"] = {"fused_kernel": {"fp64_slots": slots, "hbm_bytes": out_bytes}}
     c["hbm_bytes"] = out_bytes
@@ -452,7 +459,7 @@ class Bench:
                  "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
                  "peak_source": ("DFMA issue rate measured in this run by plogp_fp64_fma_rate, of measured (nominal %.2f T/s = 148 SMs x 64 lanes x 1.965 GHz)"
                                  % (NOMINAL_FP64_FMA_RATE / 1e12)) if alu else "HBM copy bandwidth, of %s" % self.peak_src}
-            if alu and name in ("sweep_kernel", "decide_kernel"):
+            if alu and name in ("sweep_kernel", "decide_kernel", "segmin_kernel"):
                 # stricter accounting: the compare of a segmented cell runs in the integer pipe, so only its DFMA
                 # is an FP64 slot (1 instead of 2 per segmented cell)
                 strict = (work["fp64_slots"] - seg_cells) * per_launch

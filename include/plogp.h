@@ -275,7 +275,8 @@ enum {
     PLOGP_KERNEL_DECIDE = 3,       /* Broadcast decision, lanes <-> P (short candidate lists) */
     PLOGP_KERNEL_SCATTER = 4,      /* Scatter decision */
     PLOGP_KERNEL_ENVELOPE = 5,     /* segment search by lower envelope (search_mode 1) */
-    PLOGP_N_KERNEL_KINDS = 6
+    PLOGP_KERNEL_SEGMIN = 6,       /* segmented minima of plogp_predict, lanes <-> P (short candidate lists) */
+    PLOGP_N_KERNEL_KINDS = 7
 };
 int plogp_profile_enable(plogp_tables *tables, int enable);
 int plogp_profile_read(plogp_tables *tables, double *ms, int32_t *launches);

@@ -459,6 +459,20 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             g_launches += 1;
         }
         GridDev Gf = pl.G;
+        if (predict && pl.inline_sweep && pl.n_seg > 0) {
+            // Predictions on short candidate lists: the segmented minima (planes 2, 5, 9 and the best segment sizes)
+            // come from the lane<->P kernel; fused_kernel then writes the closed-form planes only.
+            SegminParams sp{};
+            sp.T = h->T; sp.G = pl.G;
+            sp.n_mgroups = (pl.G.n_m + kSegMG - 1) / kSegMG; sp.n_ptiles = (pl.G.n_P + kSegTileP - 1) / kSegTileP;
+            sp.table0 = t0; sp.n_tables_launch = nt; sp.out_table0 = out.out_table0;
+            sp.p_time = out.p_time; sp.p_best_s = out.p_best_s;
+            { LaunchTimer lt(h, PLOGP_KERNEL_SEGMIN, st); CK(launch_segmin(sp, st)); }
+            g_launches += 1;
+            Gf.mask &= ~kSegBits;
+            Gf.n_s = 0;
+            if (!Gf.mask) continue;
+        }
         if (use_decide) {
             // Broadcast half with lanes <-> P; the Scatter half (no candidate lists) follows in fused_kernel.
             DecideParams dp{};

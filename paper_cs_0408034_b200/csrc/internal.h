@@ -137,6 +137,21 @@ constexpr int kDecTileP = 32 * kDecR;                  // 256 process counts per
 constexpr int kDecMG = 16;                             // message sizes per CTA (at most), split over the warps
 constexpr int kDecU = 4;                               // list entries per filter test
 
+// segmin_kernel (segmented minima of plogp_predict on short candidate lists, lanes <-> P): see segmin.cu
+struct SegminParams {
+    TableDev T;
+    GridDev G;
+    int n_mgroups, n_ptiles;
+    int table0, n_tables_launch, out_table0;
+    double *p_time;      // [n_tables][13][n_P][n_m]: planes 2, 5, 9 are written
+    uint32_t *p_best_s;  // [n_tables][3][n_P][n_m], or nullptr
+};
+constexpr int kSegThreads = 128;
+constexpr int kSegWarps = kSegThreads / 32;
+constexpr int kSegR = 8;                 // process counts per thread
+constexpr int kSegTileP = 32 * kSegR;    // process counts per CTA
+constexpr int kSegMG = 8;                // message sizes per CTA, two per warp
+
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kFusedR = 4;   // process counts per thread and pass in the fused kernel
@@ -153,6 +168,8 @@ cudaError_t launch_s1_tiles(const S1Params &p, cudaStream_t st);
 size_t decide_smem_bytes(const TableDev &T, const GridDev &G);
 cudaError_t launch_decide(const DecideParams &p, cudaStream_t st);
 cudaError_t launch_fp64_probe(double *d_sink, int iters, int blocks, cudaStream_t st);
+size_t segmin_smem_bytes(const TableDev &T, const GridDev &G);
+cudaError_t launch_segmin(const SegminParams &p, cudaStream_t st);
 cudaError_t launch_barrier(const TableDev &T, const GridDev &G, int table0, int n_tables_launch, uint8_t *d_strategy, uint32_t *d_sbytes,
                            double *d_time, cudaStream_t st);
 cudaError_t launch_surface(const SensParams &p, cudaStream_t st);
