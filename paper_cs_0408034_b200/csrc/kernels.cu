@@ -14,8 +14,10 @@
 //                  the predicted planes or the decision table.  The general path.
 //   s1_tile_sum    per-tile and per-warp-run sums for the Scatter Chain sum when P is split over CTAs
 //                  (reduce-then-scan: the consumers add up the sums of the tiles in front of theirs).
-// The decision table of short candidate lists has faster, specialised kernels in decide.cu
-// (Broadcast half) and scatter.cu (Scatter half).
+// Short candidate lists have faster, specialised kernels: decide.cu (Broadcast half of the decision
+// table), scatter.cu (Scatter half), segmin.cu (segmented planes of the predictions); the host routes
+// them there, so fused_kernel's own inline loop over short lists only serves callers of launch_fused
+// that pass segmented strategies without partial minima.
 #include "device_common.cuh"
 
 namespace plogp {
