@@ -148,7 +148,13 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
     double x = static_cast<double>(P0 - 1) * md;
 
     const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
-    size_t o = (static_cast<size_t>(table - p.out_table0) * p.om.planes + p.om.plane_scat) * plane + static_cast<size_t>(e0) * p.G.n_m + midx;
+    const size_t o = (static_cast<size_t>(table - p.out_table0) * p.om.planes + p.om.plane_scat) * plane + static_cast<size_t>(e0) * p.G.n_m + midx;
+    // running output pointers (one row of n_m cells further per process count) and the ids as the caller names them
+    double *out_t = p.d_time + o;
+    uint8_t *out_id = p.d_strategy + o;
+    uint32_t *out_s = p.d_sbytes + o;
+    const size_t row = static_cast<size_t>(p.G.n_m);
+    const uint8_t id10 = p.om.id_of[10], id11 = p.om.id_of[11], id12 = p.om.id_of[12];
     int P = P0;
     int lc = 32 - __clz(P - 1);               // ceil(log2 P)
     int P_next_lc = (1 << lc) + 1;            // first process count with a larger ceil(log2 P)
@@ -168,8 +174,8 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
             if (on12) s2 = s_cum[(lc - 1) * 32 + lane] + lcL;
         }
         double bt = CUDART_INF;
-        int bid = 255;
-        if (on10) { bt = fma(pm1, gm, L); bid = 10; }                    // Flat Tree
+        uint8_t bid = 255;
+        if (on10) { bt = fma(pm1, gm, L); bid = id10; }                  // Flat Tree
         if (on11) {                                                      // Chain
             if (CONTIG) {
                 run += w.at(s_tab, npad, x);
@@ -178,13 +184,13 @@ __global__ void __launch_bounds__(kThreads, 4) scatter_kernel(const FusedParams 
                 run += listed_step(e, P, w);
             }
             const double t = fma(pm1, L, run);
-            if (t < bt) { bt = t; bid = 11; }
+            if (t < bt) { bt = t; bid = id11; }
         }
-        if (on12 && s2 < bt) { bt = s2; bid = 12; }                      // Binomial Tree
-        p.d_time[o] = bt;
-        p.d_strategy[o] = bid < 16 ? p.om.id_of[bid] : static_cast<uint8_t>(bid);
-        p.d_sbytes[o] = 0u;
-        o += p.G.n_m;
+        if (on12 && s2 < bt) { bt = s2; bid = id12; }                    // Binomial Tree
+        *out_t = bt;
+        *out_id = bid;
+        *out_s = 0u;
+        out_t += row; out_id += row; out_s += row;
         if (CONTIG) { ++P; pm1 += 1.0; }
     }
 }
