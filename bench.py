@@ -85,7 +85,10 @@ def work_counts(w):
         per_kernel["fused_kernel"] = {"fp64_slots": len(unseg_b) * cells_pm + scat_slots, "hbm_bytes": 13 * (bcast_dec + scat_dec)}
     else:
         if seg_ids:
-            per_kernel["decide_kernel"] = {"fp64_slots": 2 * seg_cells + len(unseg_b) * cells_pm, "hbm_bytes": 13 * bcast_dec}
+            # selection_slots: the strategy-selection compares per decision cell (enabled Broadcast strategies - 1), which
+            # the per-unit table of the roofline also lists as FP64 work; reported beside `frac`, not inside it
+            per_kernel["decide_kernel"] = {"fp64_slots": 2 * seg_cells + len(unseg_b) * cells_pm, "hbm_bytes": 13 * bcast_dec,
+                                           "selection_slots": (len(seg_ids) + len(unseg_b) - 1) * cells_pm}
             if scat:
                 per_kernel["scatter_kernel"] = {"fp64_slots": scat_slots, "hbm_bytes": 13 * scat_dec}
         elif unseg_b:
@@ -459,6 +462,8 @@ class Bench:
                  "alu_time_ms": t_alu * 1e3, "hbm_time_ms": t_hbm * 1e3,
                  "peak_source": ("DFMA issue rate measured in this run by plogp_fp64_fma_rate, of measured (nominal %.2f T/s = 148 SMs x 64 lanes x 1.965 GHz)"
                                  % (NOMINAL_FP64_FMA_RATE / 1e12)) if alu else "HBM copy bandwidth, of %s" % self.peak_src}
+            if alu and work.get("selection_slots"):
+                r["frac_with_selection_compares"] = max((slots + work["selection_slots"] * per_launch) / fma_rate, t_hbm) / dur
             if alu and name in ("sweep_kernel", "decide_kernel", "segmin_kernel"):
                 # stricter accounting: the compare of a segmented cell runs in the integer pipe, so only its DFMA
                 # is an FP64 slot (1 instead of 2 per segmented cell)
