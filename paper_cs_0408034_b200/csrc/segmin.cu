@@ -32,6 +32,7 @@ constexpr int kIntMax = 0x7FFFFFFF;
 constexpr int kStride = kSegTileP + 1;   // doubles per staged row: the transposed reads stay conflict-free
 constexpr int kIStride = kSegTileP + 2;  // 16-bit candidate indices per staged row
 constexpr uint32_t kWhole = 0xFFFEu;     // no candidate fits: the whole message in one segment
+static_assert(kMaxInlineS <= 64, "warp_argmin_pilot keeps a candidate index in six bits");
 
 struct SegSmem {
     double *tab, *gs, *gm, *lf, *lc, *pm1, *lq, *st_time;
@@ -64,6 +65,16 @@ __host__ __device__ inline size_t seg_layout(int npad, int n_s, unsigned char *b
 }
 
 __device__ __forceinline__ int hi32(double x) { return __double2hiint(x); }
+
+// Index (< 64) of a smallest non-negative value over the warp, up to the last 6 bits of its low word: two integer
+// warp reductions (high word, then low word with the index in its last bits).  Good enough for a pilot: the sweep's
+// exact comparisons settle what the pilot leaves open.
+__device__ __forceinline__ int warp_argmin_pilot(double v, int idx)
+{
+    const int hmin = __reduce_min_sync(0xffffffffu, hi32(v));
+    const unsigned key = hi32(v) == hmin ? ((static_cast<unsigned>(__double2loint(v)) & ~0x3Fu) | static_cast<unsigned>(idx & 0x3F)) : 0xFFFFFFFFu;
+    return static_cast<int>(__reduce_min_sync(0xffffffffu, key) & 0x3Fu);
+}
 
 __device__ __forceinline__ void offer(double &bt, uint32_t &bidx, double t, uint32_t idx)
 {
@@ -149,8 +160,8 @@ __global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminPara
             lq[c] = Q;
             l5[c] = make_double2(B, C);
         }
-        warp_min_pair(qb, qc);  // smallest Q, smallest candidate on ties: the winner of ids 2 and 9 for every P
-        warp_min_pair(tb, tc);  // id 5's winner at the middle of the tile
+        qc = warp_argmin_pilot(qb, qc);  // smallest Q: the winner of ids 2 and 9 for every P
+        tc = warp_argmin_pilot(tb, tc);  // id 5's winner at the middle of the tile
         __syncwarp();
         // the pilots leave the lists (their own cells would always pass the filter); the running minima start from them
         const double q_pilot = lq[qc];
