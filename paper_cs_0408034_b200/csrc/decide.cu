@@ -23,7 +23,11 @@
 // which some cell can reach the minimum is re-evaluated with the exact FP64 comparison, for the
 // eight-cell rows that need it.  With a good pilot that is rare.
 //
-// Results are staged in shared memory as [m][P] and written out as rows of consecutive m.
+// Once started, the running minima (time and winner code) live in shared memory as [m][P], which is
+// also the staging layout of the write-out: the loops keep only minus their high words in registers,
+// the exact pass reads and writes the minima themselves.  The codes carry the strategy ids as the
+// caller names them (OutMap::id_of keeps their order), so the write-out, rows of consecutive m per
+// process count, only has to split a code into its id and its segment size.
 #include "device_common.cuh"
 
 #include <algorithm>
@@ -46,7 +50,7 @@ constexpr int kIntMax = 0x7FFFFFFF;
 struct DecSmem {
     double *tab, *gs, *gm, *lf, *lc, *pm1, *l2, *st_time;
     double2 *l1;
-    uint32_t *sval;
+    uint32_t *sval;   // [256]: segment sizes by candidate index; [kCandNone] = 0
     uint16_t *c1, *c2, *st_code;
     int cap1, cap2;
 };
@@ -60,7 +64,7 @@ __host__ __device__ inline size_t dec_layout(int npad, int n_s, unsigned char *b
     const int cap1 = round_up(2 * nsv + 4, U), cap2 = round_up(nsv + 1, U);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off += (bytes + 15) & ~size_t(15); return at; };
-    const size_t o_tab = take(3 * size_t(npad) * 8), o_gs = take(size_t(nsv) * 8), o_sv = take(size_t(nsv) * 4),
+    const size_t o_tab = take(3 * size_t(npad) * 8), o_gs = take(size_t(nsv) * 8), o_sv = take(256 * 4),
                  o_gm = take(kDecMG * 8), o_lf = take(kDecTileP * 8), o_lc = take(kDecTileP * 8), o_pm = take(kDecTileP * 8),
                  o_l1 = take(size_t(kDecWarps) * cap1 * 16), o_l2 = take(size_t(kDecWarps) * cap2 * 8),
                  o_c1 = take(size_t(kDecWarps) * cap1 * 2), o_c2 = take(size_t(kDecWarps) * cap2 * 2),
@@ -128,6 +132,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
         sm.sval[si] = s;
         sm.gs[si] = gap_at(sm.tab, npad, static_cast<double>(s));
     }
+    if (tid == 0) sm.sval[kCandNone] = 0u;
     if (tid >= kDecThreads - kDecMG) {  // g(m) of the group's message sizes, by the last threads
         const int mi = tid - (kDecThreads - kDecMG);
         if (mi < n_mi) sm.gm[mi] = gap_at(sm.tab, npad, static_cast<double>(p.G.m_list[m0 + mi]));
@@ -144,6 +149,9 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     const double x2_mid = static_cast<double>(31 - __clz(P_mid));
     const double c2_mid = static_cast<double>(32 - __clz(P_mid - 1)) * L;
 
+    // the codes carry the strategy ids as the caller names them (the relabelling keeps their order)
+    auto idc = [&](int id) { return static_cast<uint32_t>(p.om.id_of[id]) << 8; };
+    const uint32_t code2 = idc(2), code5 = idc(5), code9 = idc(9);
     const uint32_t un = mask & 0x1Bu;  // unsegmented members of the P list: ids 0, 1, 3, 4
     const int n_un = __popc(un);
     const bool has2 = (mask >> 2) & 1u, has5 = (mask >> 5) & 1u, has6 = (mask >> 6) & 1u, has7 = (mask >> 7) & 1u,
@@ -204,13 +212,13 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 const double a = id >= 3 ? gm + (id == 4 ? rdv : L) : gm;
                 const double c = id >= 3 ? 0.0 : (id == 1 ? rdv : L);
                 l1[pos] = make_double2(a, c);
-                c1[pos] = static_cast<uint16_t>((id << 8) | kCandNone);
+                c1[pos] = static_cast<uint16_t>(idc(id) | kCandNone);
                 pilot_offer(fma(x1_mid, a, c), pos);
             }
         }
         if (lane == 4 && has7) {  // Binomial Tree
             l2[0] = gm;
-            c2[0] = static_cast<uint16_t>((7u << 8) | kCandNone);
+            c2[0] = static_cast<uint16_t>(idc(7) | kCandNone);
             pilot_offer(fma(x2_mid, gm, c2_mid), 256u);
         }
         for (int i = n1 + lane; i < n1p; i += 32) {  // padding never reaches the minimum
@@ -235,18 +243,18 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             const int pq = env ? 0 : c, p5 = env ? c - lo5 : c;  // positions inside the strategies' parts of the lists
             if (has2 && in_q) {  // (P-1) (g(s) k) + L
                 l1[o2 + pq] = make_double2(Q, L);
-                c1[o2 + pq] = static_cast<uint16_t>((2u << 8) | cand);
+                c1[o2 + pq] = static_cast<uint16_t>(code2 | cand);
                 pilot_offer(fma(x1_mid, Q, L), o2 + pq);
             }
             if (has5 && in_5) {  // (P-1) (g(s) + L) + g(s) (k-1)
                 const double B = gsv + L, C = gsv * (k - 1.0);
                 l1[o5 + p5] = make_double2(B, C);
-                c1[o5 + p5] = static_cast<uint16_t>((5u << 8) | cand);
+                c1[o5 + p5] = static_cast<uint16_t>(code5 | cand);
                 pilot_offer(fma(x1_mid, B, C), o5 + p5);
             }
             if (has9 && in_q) {  // floor(log2 P) g(s) k + ceil(log2 P) L
                 l2[o9 + pq] = Q;
-                c2[o9 + pq] = static_cast<uint16_t>((9u << 8) | cand);
+                c2[o9 + pq] = static_cast<uint16_t>(code9 | cand);
                 pilot_offer(fma(x2_mid, Q, c2_mid), 256u + o9 + pq);
             }
         }
@@ -302,16 +310,28 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             double t[R];
 #pragma unroll
             for (int r = 0; r < R; ++r) t[r] = lcL[r] * w;
-            single((6u << 8) | kCandNone, t);
+            single(idc(6) | kCandNone, t);
         }
         if (has8) {  // Binomial Tree Rendezvous: floor(log2 P) g(m) + ceil(log2 P) rdv
             double t[R];
 #pragma unroll
             for (int r = 0; r < R; ++r) t[r] = fma(lf[r], gm, lcL[r] * rdv);
-            single((8u << 8) | kCandNone, t);
+            single(idc(8) | kCandNone, t);
         }
+        // from here on the running minima live in shared memory (the staging area of the write-out): the loops only need
+        // minus their high words, and only the exact pass touches the minima themselves.  (The plain add-then-min form
+        // below is left to the compiler on purpose: it splits the work between two pipes and measured faster than the
+        // fused add-min instruction.)
+        double *st = sm.st_time + mi * kStageStride + lane;
+        uint16_t *sc = sm.st_code + mi * kCodeStride + lane;
+        int nhb[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) lcL[r] *= L;
+        for (int r = 0; r < R; ++r) {
+            lcL[r] *= L;
+            nhb[r] = -hi32(bt[r]);
+            st[32 * r] = bt[r];
+            sc[32 * r] = static_cast<uint16_t>(bcode[r]);
+        }
 
         // The filter of a group of U list entries: every cell is evaluated (one DFMA each); per process
         // count the smallest high word of the U times minus the high word of the running minimum says
@@ -329,16 +349,21 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             for (int r = 0; r < R; ++r) {
                 const int h0 = hi32(fma(lf[r], q01.x, lcL[r])), h1 = hi32(fma(lf[r], q01.y, lcL[r]));
                 const int h2 = hi32(fma(lf[r], q23.x, lcL[r])), h3 = hi32(fma(lf[r], q23.y, lcL[r]));
-                acc = min(acc, min(min(h0, h1), min(h2, h3)) - hi32(bt[r]));
+                acc = min(acc, min(min(h0, h1), min(h2, h3)) + nhb[r]);
             }
             if (__any_sync(kFull, acc <= 0)) {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
                     const int h0 = hi32(fma(lf[r], q01.x, lcL[r])), h1 = hi32(fma(lf[r], q01.y, lcL[r]));
                     const int h2 = hi32(fma(lf[r], q23.x, lcL[r])), h3 = hi32(fma(lf[r], q23.y, lcL[r]));
-                    if (__any_sync(kFull, min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]))) {
+                    if (__any_sync(kFull, min(min(h0, h1), min(h2, h3)) + nhb[r] <= 0)) {
+                        double b = st[32 * r];
+                        uint32_t code = sc[32 * r];
 #pragma unroll 1
-                        for (int u = 0; u < U; ++u) offer(bt[r], bcode[r], fma(lf[r], l2[j + u], lcL[r]), c2[j + u]);
+                        for (int u = 0; u < U; ++u) offer(b, code, fma(lf[r], l2[j + u], lcL[r]), c2[j + u]);
+                        st[32 * r] = b;
+                        sc[32 * r] = static_cast<uint16_t>(code);
+                        nhb[r] = -hi32(b);
                     }
                 }
             }
@@ -356,53 +381,59 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             for (int r = 0; r < R; ++r) {
                 const int h0 = hi32(fma(pm1[r], e0.x, e0.y)), h1 = hi32(fma(pm1[r], e1.x, e1.y));
                 const int h2 = hi32(fma(pm1[r], e2.x, e2.y)), h3 = hi32(fma(pm1[r], e3.x, e3.y));
-                acc = min(acc, min(min(h0, h1), min(h2, h3)) - hi32(bt[r]));
+                acc = min(acc, min(min(h0, h1), min(h2, h3)) + nhb[r]);
             }
             if (__any_sync(kFull, acc <= 0)) {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
                     const int h0 = hi32(fma(pm1[r], e0.x, e0.y)), h1 = hi32(fma(pm1[r], e1.x, e1.y));
                     const int h2 = hi32(fma(pm1[r], e2.x, e2.y)), h3 = hi32(fma(pm1[r], e3.x, e3.y));
-                    if (__any_sync(kFull, min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]))) {
+                    if (__any_sync(kFull, min(min(h0, h1), min(h2, h3)) + nhb[r] <= 0)) {
+                        double b = st[32 * r];
+                        uint32_t code = sc[32 * r];
 #pragma unroll 1
                         for (int u = 0; u < U; ++u) {
                             const double2 e = l1[j + u];
-                            offer(bt[r], bcode[r], fma(pm1[r], e.x, e.y), c1[j + u]);
+                            offer(b, code, fma(pm1[r], e.x, e.y), c1[j + u]);
                         }
+                        st[32 * r] = b;
+                        sc[32 * r] = static_cast<uint16_t>(code);
+                        nhb[r] = -hi32(b);
                     }
                 }
             }
         }
 
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            sm.st_time[mi * kStageStride + 32 * r + lane] = bt[r];
-            sm.st_code[mi * kCodeStride + 32 * r + lane] = static_cast<uint16_t>(bcode[r]);
-        }
     }
     __syncthreads();
 
-    // transposed write-out of the staged group: rows of p.mg consecutive m per process count
+    // transposed write-out of the staged group: rows of p.mg consecutive m per process count, running pointers
     if (p.vec_out) {
         // two message sizes per lane: 16-byte, 8-byte and 2-byte stores (the host has checked the alignment)
         const int half = p.mg >> 1;
-        const int mi = 2 * (lane & (half - 1)), prow = lane / half, rows = 32 / half;
+        const int mi = 2 * (lane & (half - 1)), rows = 32 / half, pr0 = warp * rows + lane / half, prs = kDecWarps * rows;
         if (mi < n_mi) {
             const uint32_t m_u0 = p.G.m_list[m0 + mi], m_u1 = p.G.m_list[m0 + mi + 1];
             const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
-            const size_t base = (static_cast<size_t>(table - p.out_table0) * p.om.planes + p.om.plane_bcast) * plane + static_cast<size_t>(m0 + mi);
-            const double *st0 = sm.st_time + mi * kStageStride, *st1 = st0 + kStageStride;
-            const uint16_t *sc0 = sm.st_code + mi * kCodeStride, *sc1 = sc0 + kCodeStride;
-            for (int pr = warp * rows + prow; pr < n_valid; pr += kDecWarps * rows) {
-                const size_t o = base + static_cast<size_t>(tile0 + pr) * p.G.n_m;
-                const uint32_t code0 = sc0[pr], code1 = sc1[pr];
+            const size_t o = (static_cast<size_t>(table - p.out_table0) * p.om.planes + p.om.plane_bcast) * plane +
+                             static_cast<size_t>(tile0 + pr0) * p.G.n_m + static_cast<size_t>(m0 + mi);
+            const size_t step = static_cast<size_t>(prs) * p.G.n_m;
+            double *out_t = p.d_time + o;
+            uint32_t *out_s = p.d_sbytes + o;
+            uint8_t *out_id = p.d_strategy + o;
+            const double *st0 = sm.st_time + mi * kStageStride + pr0, *st1 = st0 + kStageStride;
+            const uint16_t *sc0 = sm.st_code + mi * kCodeStride + pr0, *sc1 = sc0 + kCodeStride;
+            for (int pr = pr0; pr < n_valid; pr += prs) {
+                const uint32_t code0 = *sc0, code1 = *sc1;
                 const uint32_t cand0 = code0 & 255u, cand1 = code1 & 255u;
-                const uint32_t s0 = cand0 == kCandNone ? 0u : (cand0 == kCandWhole ? m_u0 : sm.sval[cand0]);
-                const uint32_t s1 = cand1 == kCandNone ? 0u : (cand1 == kCandWhole ? m_u1 : sm.sval[cand1]);
-                *reinterpret_cast<double2 *>(p.d_time + o) = make_double2(st0[pr], st1[pr]);
-                *reinterpret_cast<uint2 *>(p.d_sbytes + o) = make_uint2(s0, s1);
-                *reinterpret_cast<uint16_t *>(p.d_strategy + o) =
-                    static_cast<uint16_t>(p.om.id_of[(code0 >> 8) & 15u] | (static_cast<uint32_t>(p.om.id_of[(code1 >> 8) & 15u]) << 8));
+                uint32_t s0 = sm.sval[cand0], s1 = sm.sval[cand1];
+                if (cand0 == kCandWhole) s0 = m_u0;
+                if (cand1 == kCandWhole) s1 = m_u1;
+                *reinterpret_cast<double2 *>(out_t) = make_double2(*st0, *st1);
+                *reinterpret_cast<uint2 *>(out_s) = make_uint2(s0, s1);
+                *reinterpret_cast<uint16_t *>(out_id) = static_cast<uint16_t>(__byte_perm(code0, code1, 0x0051));
+                out_t += step; out_s += step; out_id += step;
+                st0 += prs; st1 += prs; sc0 += prs; sc1 += prs;
             }
         }
     } else {
@@ -416,8 +447,8 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
                 const uint32_t code = sm.st_code[mi * kCodeStride + pr];
                 const uint32_t cand = code & 255u;
                 p.d_time[o] = sm.st_time[mi * kStageStride + pr];
-                p.d_strategy[o] = p.om.id_of[(code >> 8) & 15u];
-                p.d_sbytes[o] = cand == kCandNone ? 0u : (cand == kCandWhole ? m_u : sm.sval[cand]);
+                p.d_strategy[o] = static_cast<uint8_t>(code >> 8);
+                p.d_sbytes[o] = cand == kCandWhole ? m_u : sm.sval[cand];
             }
         }
     }
