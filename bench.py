@@ -447,7 +447,7 @@ class Bench:
             # the launching stream during the timed region)
             work = counts["per_kernel"].get(name)
             if work is None or n_launch == 0:
-                return {"kernel": name, "launches": n_launch, "ms_total": ms_total}
+                return {"kernel": name, "launches": n_launch, "ms_total": ms_total, "avg_ms": ms_total / max(n_launch, 1)}
             per_launch = steps / n_launch  # a kernel launched once per step does one step's work
             dur = ms_total / n_launch * 1e-3
             slots, nbytes = work["fp64_slots"] * per_launch, work["hbm_bytes"] * per_launch

@@ -276,7 +276,8 @@ enum {
     PLOGP_KERNEL_SCATTER = 4,      /* Scatter decision */
     PLOGP_KERNEL_ENVELOPE = 5,     /* segment search by lower envelope (search_mode 1) */
     PLOGP_KERNEL_SEGMIN = 6,       /* segmented minima of plogp_predict, lanes <-> P (short candidate lists) */
-    PLOGP_N_KERNEL_KINDS = 7
+    PLOGP_KERNEL_GAPS = 7,         /* g(1), g(s), g(m) once per table, in front of the lanes <-> P kernels on large grids */
+    PLOGP_N_KERNEL_KINDS = 8
 };
 int plogp_profile_enable(plogp_tables *tables, int enable);
 int plogp_profile_read(plogp_tables *tables, double *ms, int32_t *launches);

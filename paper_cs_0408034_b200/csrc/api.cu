@@ -70,6 +70,10 @@ struct Plan {
     size_t off_pair_m = 0, off_pair_chunk = 0, off_pair_row = 0, off_pair_base = 0;
     int tables_per_batch = 0;
     size_t scratch_bytes = 0;
+    size_t off_k = 0;          // k table of the lane <-> P kernels inside the grid blob
+    bool use_gaps = false;     // run the gap pre-pass in front of the lane <-> P kernels
+    int gaps_stride = 0;       // doubles per table in its output
+    size_t gaps_bytes_per_table = 0;
 };
 
 }  // namespace
@@ -301,6 +305,21 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
         off_s = append_aligned(blob, s32);
     }
 
+    // Short candidate lists (lane <-> P kernels): Section 2's k for every (m, candidate), as the doubles the kernels multiply with
+    const bool short_lists = pl.inline_sweep && pl.n_seg > 0 && n_s > 0;
+    if (short_lists) {
+        std::vector<double> kt(size_t(n_m) * n_s, 1.0);
+        for (int i = 0; i < n_m; ++i) {
+            const uint64_t m = g->m[i];
+            for (int c = 0; c < ns_of_m[i]; ++c) {
+                const uint64_t sv = g->s ? g->s[c] : g->s_lo + uint64_t(c) * g->s_step;
+                const uint64_t q = m / sv;
+                kt[size_t(i) * n_s + c] = double(q + ((g->k_mode == 0 && q * sv != m) ? 1 : 0));
+            }
+        }
+        pl.off_k = append_aligned(blob, kt);
+    }
+
     // ---- sweep kernel plan: (m, chunk) pairs, heaviest first ----
     if (pl.envelope) {
         // one scratch row per message size
@@ -357,6 +376,7 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     G.s_lo = uint32_t(g->s_lo);
     G.s_step = uint32_t(g->s_step);
     G.ns_of_m = reinterpret_cast<const int32_t *>(h->d_grid + off_ns);
+    G.k_list = short_lists ? reinterpret_cast<const double *>(h->d_grid + pl.off_k) : nullptr;
     G.mask = g->strategy_mask;
     G.k_mode = g->k_mode;
     G.lc_max = std::max(1, ceil_log2(P_hi));
@@ -367,11 +387,21 @@ int prepare(plogp_tables *h, const plogp_grid *g, cudaStream_t st)
     if (!pl.inline_sweep) per_table += size_t(pl.n_seg) * pl.n_pairs * n_P * (sizeof(double) + sizeof(uint32_t)) + 512;
     if (s1_on && pl.n_ptiles > 1) pl.carry_bytes_per_table = size_t(pl.n_ptiles) * (kWarps + 1) * n_m * sizeof(double);
     per_table += pl.carry_bytes_per_table;
+    // The gap pre-pass costs a launch: taken where the lane <-> P kernels run many CTAs per table and fill the GPU several times over
+    if (pl.inline_sweep && pl.n_seg > 0) {
+        const long long ctas_per_table = (long long)pl.dec_mgroups * pl.dec_ptiles;
+        pl.use_gaps = ctas_per_table >= 4 && ctas_per_table * h->T.n_tables >= (long long)h->sm_count * 16;
+        if (pl.use_gaps) {
+            pl.gaps_stride = (1 + n_s + n_m + 1) & ~1;
+            pl.gaps_bytes_per_table = size_t(pl.gaps_stride) * sizeof(double);
+            per_table += pl.gaps_bytes_per_table;
+        }
+    }
     pl.tables_per_batch = h->T.n_tables;
     if (!pl.inline_sweep && per_table * h->T.n_tables > kSweepScratchLimit)
         pl.tables_per_batch = int(std::max<size_t>(1, kSweepScratchLimit / per_table));
     pl.tables_per_batch = std::min(pl.tables_per_batch, 65535);
-    pl.scratch_bytes = per_table ? per_table * pl.tables_per_batch + 256 : 0;
+    pl.scratch_bytes = per_table ? per_table * pl.tables_per_batch + 1024 : 0;  // the sections start on 256-byte boundaries
     if (pl.scratch_bytes > h->ws_cap) {
         if (h->d_ws) CK(cudaFree(h->d_ws));
         h->d_ws = nullptr;
@@ -429,7 +459,19 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             part_idx = reinterpret_cast<uint32_t *>(ws);
             ws += align_up(cells * sizeof(uint32_t), 256);
         }
-        if (need_carry) tile_sum = reinterpret_cast<double *>(ws);
+        if (need_carry) {
+            tile_sum = reinterpret_cast<double *>(ws);
+            ws += align_up(pl.carry_bytes_per_table * nt, 256);
+        }
+        double *gaps = nullptr;
+        if (pl.use_gaps && pl.inline_sweep && pl.n_seg > 0 && (predict || use_decide)) {
+            gaps = reinterpret_cast<double *>(ws);
+            GapsParams gp{};
+            gp.T = h->T; gp.G = pl.G;
+            gp.table0 = t0; gp.n_tables_launch = nt; gp.gaps = gaps; gp.stride = pl.gaps_stride;
+            { LaunchTimer lt(h, PLOGP_KERNEL_GAPS, st); CK(launch_gaps(gp, st)); }
+            g_launches += 1;
+        }
 
         if (pl.envelope) {
             EnvParams ep{};
@@ -467,6 +509,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             sp.n_mgroups = (pl.G.n_m + kSegMG - 1) / kSegMG; sp.n_ptiles = (pl.G.n_P + kSegTileP - 1) / kSegTileP;
             sp.table0 = t0; sp.n_tables_launch = nt; sp.out_table0 = out.out_table0;
             sp.p_time = out.p_time; sp.p_best_s = out.p_best_s;
+            sp.gaps = gaps; sp.gaps_stride = pl.gaps_stride;
             { LaunchTimer lt(h, PLOGP_KERNEL_SEGMIN, st); CK(launch_segmin(sp, st)); }
             g_launches += 1;
             Gf.mask &= ~kSegBits;
@@ -482,6 +525,7 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             dp.table0 = t0; dp.n_tables_launch = nt; dp.out_table0 = out.out_table0; dp.om = out.om;
             dp.d_strategy = out.d_strategy; dp.d_sbytes = out.d_sbytes; dp.d_time = out.d_time;
             dp.envelope = pl.envelope_short ? 1 : 0;
+            dp.gaps = gaps; dp.gaps_stride = pl.gaps_stride;
             dp.vec_out = (pl.G.n_m % 2 == 0) && pl.dec_mg >= 2 && reinterpret_cast<uintptr_t>(out.d_time) % 16 == 0 &&
                          reinterpret_cast<uintptr_t>(out.d_sbytes) % 8 == 0 && reinterpret_cast<uintptr_t>(out.d_strategy) % 2 == 0;
             { LaunchTimer lt(h, PLOGP_KERNEL_DECIDE, st); CK(launch_decide(dp, st)); }

@@ -117,7 +117,9 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     const int tile0 = ptile * kDecTileP;
     const int n_valid = min(kDecTileP, p.G.n_P - tile0);
 
-    stage_table(sm.tab, p.T, table);
+    // g at the kernel's arguments: read from the gap pre-pass where the host has run it, else interpolated here
+    const double *grow = p.gaps ? p.gaps + static_cast<size_t>(trel) * p.gaps_stride : nullptr;
+    if (!grow) stage_table(sm.tab, p.T, table);
     // floor(log2 P) and ceil(log2 P) of the tile's process counts, as doubles
     for (int i = tid; i < kDecTileP; i += kDecThreads) {
         const int P = P_at(p.G, min(tile0 + i, p.G.n_P - 1));
@@ -130,14 +132,14 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     for (int si = tid; si < p.G.n_s; si += kDecThreads) {
         const uint32_t s = s_at(p.G, si);
         sm.sval[si] = s;
-        sm.gs[si] = gap_at(sm.tab, npad, static_cast<double>(s));
+        sm.gs[si] = grow ? grow[1 + si] : gap_at(sm.tab, npad, static_cast<double>(s));
     }
     if (tid == 0) sm.sval[kCandNone] = 0u;
     if (tid >= kDecThreads - kDecMG) {  // g(m) of the group's message sizes, by the last threads
         const int mi = tid - (kDecThreads - kDecMG);
-        if (mi < n_mi) sm.gm[mi] = gap_at(sm.tab, npad, static_cast<double>(p.G.m_list[m0 + mi]));
+        if (mi < n_mi) sm.gm[mi] = grow ? grow[1 + p.G.n_s + m0 + mi] : gap_at(sm.tab, npad, static_cast<double>(p.G.m_list[m0 + mi]));
     }
-    const double g1 = gap_at(sm.tab, npad, 1.0);
+    const double g1 = grow ? grow[0] : gap_at(sm.tab, npad, 1.0);
     const double rdv = 2.0 * g1 + 3.0 * L;  // rendezvous handshake: 2 g(1) + 3 L
     __syncthreads();
 
@@ -162,10 +164,10 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
 
     for (int mi = warp; mi < n_mi; mi += kDecWarps) {
         const int midx = m0 + mi;
-        const uint32_t m_u = p.G.m_list[midx];
         const int ns = p.G.ns_of_m[midx];
         const int nsv = max(ns, 1);  // candidates actually evaluated (none fits: the whole message, k = 1)
         const double gm = sm.gm[mi];
+        const double *krow = p.G.k_list + static_cast<size_t>(midx) * p.G.n_s;
         // Lower-envelope search (p.envelope, tables whose gaps never decrease): ids 2 and 9 keep only the candidate
         // with the smallest g(s) k (their minimum over s for every P at once, a rounded fused multiply-add being
         // monotone in it), id 5 only the candidates between its winners at the tile's last and first process
@@ -178,7 +180,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             double qb = CUDART_INF, tf = CUDART_INF, tl = CUDART_INF;
             int qc = kIntMax, ef = kIntMax, el = kIntMax;
             for (int c = lane; c < ns; c += 32) {
-                const double gsv = sm.gs[c], k = static_cast<double>(segments(m_u, sm.sval[c], p.G.k_mode));
+                const double gsv = sm.gs[c], k = krow[c];
                 const double Q = gsv * k, B = gsv + L, C = gsv * (k - 1.0);
                 if (Q < qb) { qb = Q; qc = c; }
                 const double t1 = fma(x_first, B, C), t2 = fma(x_last, B, C);
@@ -235,7 +237,7 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
             uint32_t cand = kCandWhole;
             if (ns > 0) {
                 gsv = sm.gs[c];
-                k = static_cast<double>(segments(m_u, sm.sval[c], p.G.k_mode));
+                k = krow[c];  // Section 2's k, from the host's table
                 cand = static_cast<uint32_t>(c);
             }
             const double Q = gsv * k;

@@ -38,6 +38,7 @@ struct GridDev {
     int n_s;
     uint32_t s_lo, s_step;
     const int32_t *ns_of_m;  // device [n_m]: number of candidates s <= m (0 => unsegmented fallback)
+    const double *k_list;    // device [n_m][n_s]: Section 2's k for every (m, candidate s <= m), short candidate lists only
     uint32_t mask;
     int k_mode;
     int lc_max;  // ceil(log2 P_hi)
@@ -114,10 +115,22 @@ struct S1Params {
     double *tile_sum;  // [n_tables_launch][n_ptiles][9][n_m]: the 8 warps' shares, then the tile's total
 };
 
+// Gap pre-pass (gaps.cu): g at every distinct argument of the lane <-> P kernels, once per table.
+// Row of a table: [0] = g(1), [1 .. n_s] = g(s_i), [1 + n_s .. 1 + n_s + n_m) = g(m_j).
+struct GapsParams {
+    TableDev T;
+    GridDev G;
+    int table0, n_tables_launch;
+    double *gaps;  // [n_tables_launch][stride]
+    int stride;
+};
+
 // Decision kernel for short candidate lists (lanes <-> P): see decide.cu
 struct DecideParams {
     TableDev T;
     GridDev G;
+    const double *gaps;  // rows of the gap pre-pass for this launch's tables, or nullptr: the kernel interpolates itself
+    int gaps_stride;
     int n_mgroups, n_ptiles;
     int mg;  // message sizes per CTA, 1..kDecMG
     int envelope;  // lower-envelope search: the lists keep only the candidates that can win (see decide.cu)
@@ -141,6 +154,8 @@ constexpr int kDecU = 4;                               // list entries per filte
 struct SegminParams {
     TableDev T;
     GridDev G;
+    const double *gaps;  // as in DecideParams
+    int gaps_stride;
     int n_mgroups, n_ptiles;
     int table0, n_tables_launch, out_table0;
     double *p_time;      // [n_tables][13][n_P][n_m]: planes 2, 5, 9 are written
@@ -170,6 +185,7 @@ cudaError_t launch_decide(const DecideParams &p, cudaStream_t st);
 cudaError_t launch_fp64_probe(double *d_sink, int iters, int blocks, cudaStream_t st);
 size_t segmin_smem_bytes(const TableDev &T, const GridDev &G);
 cudaError_t launch_segmin(const SegminParams &p, cudaStream_t st);
+cudaError_t launch_gaps(const GapsParams &p, cudaStream_t st);
 cudaError_t launch_barrier(const TableDev &T, const GridDev &G, int table0, int n_tables_launch, uint8_t *d_strategy, uint32_t *d_sbytes,
                            double *d_time, cudaStream_t st);
 cudaError_t launch_surface(const SensParams &p, cudaStream_t st);

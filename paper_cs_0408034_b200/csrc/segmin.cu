@@ -106,7 +106,9 @@ __global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminPara
     const int tile0 = ptile * kSegTileP;
     const int n_valid = min(kSegTileP, p.G.n_P - tile0);
 
-    stage_table(sm.tab, p.T, table);
+    // g at the kernel's arguments: read from the gap pre-pass where the host has run it, else interpolated here
+    const double *grow = p.gaps ? p.gaps + static_cast<size_t>(trel) * p.gaps_stride : nullptr;
+    if (!grow) stage_table(sm.tab, p.T, table);
     for (int i = tid; i < kSegTileP; i += kSegThreads) {
         const int P = P_at(p.G, min(tile0 + i, p.G.n_P - 1));
         sm.lf[i] = static_cast<double>(31 - __clz(P));
@@ -118,11 +120,11 @@ __global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminPara
     for (int si = tid; si < p.G.n_s; si += kSegThreads) {
         const uint32_t s = s_at(p.G, si);
         sm.sval[si] = s;
-        sm.gs[si] = gap_at(sm.tab, npad, static_cast<double>(s));
+        sm.gs[si] = grow ? grow[1 + si] : gap_at(sm.tab, npad, static_cast<double>(s));
     }
     if (tid >= kSegThreads - kSegMG) {
         const int mi = tid - (kSegThreads - kSegMG);
-        if (mi < n_mi) sm.gm[mi] = gap_at(sm.tab, npad, static_cast<double>(p.G.m_list[m0 + mi]));
+        if (mi < n_mi) sm.gm[mi] = grow ? grow[1 + p.G.n_s + m0 + mi] : gap_at(sm.tab, npad, static_cast<double>(p.G.m_list[m0 + mi]));
     }
     __syncthreads();
 
@@ -132,11 +134,11 @@ __global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminPara
 
     for (int mi = warp; mi < n_mi; mi += kSegWarps) {
         const int midx = m0 + mi;
-        const uint32_t m_u = p.G.m_list[midx];
         const int ns = p.G.ns_of_m[midx];
         const int nsv = max(ns, 1);  // candidates actually evaluated (none fits: the whole message, k = 1)
         const int np = (nsv + U - 1) / U * U;
         const double gm = sm.gm[mi];
+        const double *krow = p.G.k_list + static_cast<size_t>(midx) * p.G.n_s;
 
         // ---- coefficients of this message size (lanes <-> candidates) and the pilots ----
         __syncwarp();  // the previous message size's loops have finished reading the lists
@@ -148,7 +150,7 @@ __global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminPara
                 double gsv = gm, k = 1.0;
                 if (ns > 0) {
                     gsv = sm.gs[c];
-                    k = static_cast<double>(segments(m_u, sm.sval[c], p.G.k_mode));  // Section 2's k
+                    k = krow[c];  // Section 2's k, from the host's table
                 }
                 Q = gsv * k;
                 B = gsv + L;

@@ -281,7 +281,7 @@ def scatter_chain_static(d_sizes, d_gap, latency: float, P_lo: int, P_hi: int, d
     return out
 
 
-KERNEL_KINDS = ("sweep_kernel", "s1_tile_sum_kernel", "fused_kernel", "decide_kernel", "scatter_kernel", "envelope_kernel", "segmin_kernel")
+KERNEL_KINDS = ("sweep_kernel", "s1_tile_sum_kernel", "fused_kernel", "decide_kernel", "scatter_kernel", "envelope_kernel", "segmin_kernel", "gaps_kernel")
 
 
 def profile_enable(tables: Tables, enable: bool = True) -> None:
