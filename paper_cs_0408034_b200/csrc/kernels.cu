@@ -397,11 +397,22 @@ __global__ void __launch_bounds__(kThreads, 2) fused_kernel(const FusedParams p)
             return (static_cast<size_t>(table - p.out_table0) * planes + id_or_coll) * plane +
                    static_cast<size_t>(p0 + r) * p.G.n_m + midx;
         };
+        // Predictions: one pointer per row into the table's first plane; a strategy's plane is id * plane further on.
+        // Rows past the last process count and lanes past the last message size compute the last valid cell again
+        // (their indices are clamped), so they store the same value to the same address: no predicates on the stores.
+        unsigned char *row_t[R];
+        if (PREDICT) {
+            const size_t tab0 = static_cast<size_t>(table - p.out_table0) * 13 * plane + midx_c;
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                row_t[r] = reinterpret_cast<unsigned char *>(p.p_time + (tab0 + static_cast<size_t>(min(p0 + r, p.G.n_P - 1)) * p.G.n_m));
+        }
+        const size_t plane_bytes = plane * sizeof(double);
         auto consider = [&](int id, const double *val, const uint32_t *sval) {
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 if (PREDICT) {
-                    if (ok[r] && m_ok) p.p_time[out_index(id, 13, r)] = val[r];
+                    *reinterpret_cast<double *>(row_t[r] + id * plane_bytes) = val[r];
                 } else if (val[r] < bt[r]) {
                     bt[r] = val[r];
                     bid[r] = id;
@@ -458,14 +469,13 @@ __global__ void __launch_bounds__(kThreads, 2) fused_kernel(const FusedParams p)
                     const size_t rb = ((static_cast<size_t>(trel) * p.n_seg + slot) * p.n_pairs + row) * p.G.n_P;
 #pragma unroll
                     for (int r = 0; r < R; ++r) {
-                        if (ok[r]) {
-                            const double t = p.part_time[rb + p0 + r];
-                            if (t < st[r]) { st[r] = t; si_best[r] = p.part_idx[rb + p0 + r]; }
-                        }
+                        const int pr = min(p0 + r, p.G.n_P - 1);  // rows past the end repeat the last one
+                        const double t = p.part_time[rb + pr];
+                        if (t < st[r]) { st[r] = t; si_best[r] = p.part_idx[rb + pr]; }
                     }
                 }
 #pragma unroll
-                for (int r = 0; r < R; ++r) sb[r] = ok[r] ? s_at(p.G, static_cast<int>(si_best[r])) : 0u;
+                for (int r = 0; r < R; ++r) sb[r] = s_at(p.G, static_cast<int>(si_best[r]));
             }
             if (PREDICT && p.p_best_s) {
 #pragma unroll
