@@ -510,6 +510,8 @@ int run(plogp_tables *h, const plogp_grid *g, bool predict, FusedParams out, cud
             sp.table0 = t0; sp.n_tables_launch = nt; sp.out_table0 = out.out_table0;
             sp.p_time = out.p_time; sp.p_best_s = out.p_best_s;
             sp.gaps = gaps; sp.gaps_stride = pl.gaps_stride;
+            sp.vec_out = (pl.G.n_m % 2 == 0) && reinterpret_cast<uintptr_t>(out.p_time) % 16 == 0 &&
+                         (!out.p_best_s || reinterpret_cast<uintptr_t>(out.p_best_s) % 8 == 0);
             { LaunchTimer lt(h, PLOGP_KERNEL_SEGMIN, st); CK(launch_segmin(sp, st)); }
             g_launches += 1;
             Gf.mask &= ~kSegBits;

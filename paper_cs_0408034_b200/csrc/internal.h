@@ -156,6 +156,7 @@ struct SegminParams {
     GridDev G;
     const double *gaps;  // as in DecideParams
     int gaps_stride;
+    int vec_out;  // outputs aligned for two message sizes per store (n_m even, 16-byte aligned times, 8-byte aligned sizes)
     int n_mgroups, n_ptiles;
     int table0, n_tables_launch, out_table0;
     double *p_time;      // [n_tables][13][n_P][n_m]: planes 2, 5, 9 are written

@@ -273,13 +273,40 @@ __global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminPara
     __syncthreads();
 
     // transposed write-out: rows of 8 consecutive m per process count and strategy
-    {
+    const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
+    const int ids[3] = {2, 5, 9};
+    if (p.vec_out) {
+        // two message sizes per lane (16-byte and 8-byte stores; the host has checked the alignment), running pointers
+        constexpr int kHalf = kSegMG / 2, kRows = 32 / kHalf, kStep = kSegWarps * kRows;
+        const int mi = 2 * (lane & (kHalf - 1)), pr0 = warp * kRows + lane / kHalf;
+        if (mi < n_mi) {  // n_m is even, so mi + 1 is a message size of the grid too
+            const uint32_t m_u0 = p.G.m_list[m0 + mi], m_u1 = p.G.m_list[m0 + mi + 1];
+            const size_t cell0 = static_cast<size_t>(tile0 + pr0) * p.G.n_m + static_cast<size_t>(m0 + mi);
+            const size_t step = static_cast<size_t>(kStep) * p.G.n_m;
+#pragma unroll
+            for (int q = 0; q < 3; ++q) {
+                if (!((mask >> ids[q]) & 1u)) continue;
+                const double *st0 = sm.st_time + (q * kSegMG + mi) * kStride + pr0, *st1 = st0 + kStride;
+                const uint16_t *si0 = sm.st_idx + (q * kSegMG + mi) * kIStride + pr0, *si1 = si0 + kIStride;
+                double *out_t = p.p_time + (static_cast<size_t>(table - p.out_table0) * 13 + ids[q]) * plane + cell0;
+                uint32_t *out_s = p.p_best_s ? p.p_best_s + (static_cast<size_t>(table - p.out_table0) * 3 + q) * plane + cell0 : nullptr;
+                for (int pr = pr0; pr < n_valid; pr += kStep) {
+                    *reinterpret_cast<double2 *>(out_t) = make_double2(*st0, *st1);
+                    if (out_s) {
+                        const uint32_t i0 = *si0, i1 = *si1;
+                        *reinterpret_cast<uint2 *>(out_s) = make_uint2(i0 == kWhole ? m_u0 : sm.sval[i0], i1 == kWhole ? m_u1 : sm.sval[i1]);
+                        out_s += step;
+                    }
+                    out_t += step;
+                    st0 += kStep; st1 += kStep; si0 += kStep; si1 += kStep;
+                }
+            }
+        }
+    } else {
         const int mi = lane & (kSegMG - 1), prow = lane / kSegMG, rows = 32 / kSegMG;
         if (mi < n_mi) {
             const uint32_t m_u = p.G.m_list[m0 + mi];
-            const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
             const size_t cell0 = static_cast<size_t>(m0 + mi);
-            const int ids[3] = {2, 5, 9};
 #pragma unroll
             for (int q = 0; q < 3; ++q) {
                 if (!((mask >> ids[q]) & 1u)) continue;
