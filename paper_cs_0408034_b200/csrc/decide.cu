@@ -158,6 +158,15 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
     const int n_un = __popc(un);
     const bool has2 = (mask >> 2) & 1u, has5 = (mask >> 5) & 1u, has6 = (mask >> 6) & 1u, has7 = (mask >> 7) & 1u,
                has8 = (mask >> 8) & 1u, has9 = (mask >> 9) & 1u;
+    // The unsegmented members of the lists do not depend on the message size beyond g(m): lanes 0..3 hold ids 0, 1, 3, 4
+    // (Flat Tree (P-1) g + L, its rendezvous form (P-1) g + rdv; Chain (P-1)(g + L), rendezvous (P-1)(g + rdv)) as
+    // P-list entries (g(m) + fa, fc), lane 4 the Binomial Tree's log-list entry g(m).
+    const int fid = lane < 4 ? lane + (lane >> 1) : 7;
+    const bool f_on = lane < 5 && ((mask >> fid) & 1u);
+    const int fpos = __popc(un & ((1u << fid) - 1u));
+    const double fa = fid == 3 ? L : (fid == 4 ? rdv : 0.0);
+    const double fc = fid == 0 ? L : (fid == 1 ? rdv : 0.0);
+    const uint16_t fcode = static_cast<uint16_t>(idc(fid) | kCandNone);
     double2 *l1 = sm.l1 + warp * sm.cap1;
     double *l2 = sm.l2 + warp * sm.cap2;
     uint16_t *c1 = sm.c1 + warp * sm.cap1, *c2 = sm.c2 + warp * sm.cap2;
@@ -206,22 +215,16 @@ __global__ void __launch_bounds__(kDecThreads, 4) decide_kernel(const DecidePara
         auto pilot_offer = [&](double t, unsigned pos) {
             if (t < tb) { tb = t; pb = pos; }
         };
-        if (lane < 4) {
-            const int id = lane + (lane >> 1);  // 0, 1, 3, 4
-            if ((mask >> id) & 1u) {
-                const int pos = __popc(un & ((1u << id) - 1u));
-                // Flat Tree (P-1) g + L, its rendezvous form (P-1) g + rdv; Chain (P-1)(g + L), rendezvous (P-1)(g + rdv)
-                const double a = id >= 3 ? gm + (id == 4 ? rdv : L) : gm;
-                const double c = id >= 3 ? 0.0 : (id == 1 ? rdv : L);
-                l1[pos] = make_double2(a, c);
-                c1[pos] = static_cast<uint16_t>(idc(id) | kCandNone);
-                pilot_offer(fma(x1_mid, a, c), pos);
+        if (f_on) {  // this lane's unsegmented strategy
+            if (lane < 4) {
+                l1[fpos] = make_double2(gm + fa, fc);
+                c1[fpos] = fcode;
+                pilot_offer(fma(x1_mid, gm + fa, fc), fpos);
+            } else {
+                l2[0] = gm;
+                c2[0] = fcode;
+                pilot_offer(fma(x2_mid, gm, c2_mid), 256u);
             }
-        }
-        if (lane == 4 && has7) {  // Binomial Tree
-            l2[0] = gm;
-            c2[0] = static_cast<uint16_t>(idc(7) | kCandNone);
-            pilot_offer(fma(x2_mid, gm, c2_mid), 256u);
         }
         for (int i = n1 + lane; i < n1p; i += 32) {  // padding never reaches the minimum
             l1[i] = make_double2(CUDART_INF, CUDART_INF);
