@@ -215,6 +215,24 @@ def test_host_output_entry_point_matches_device_outputs(plogp):
     assert torch.equal(b.strategy, a.strategy.cpu()) and torch.equal(b.time.view(torch.int64), a.time.cpu().view(torch.int64))
 
 
+def test_many_tables_take_the_gap_prepass(plogp):
+    """Enough tables for the host to run gaps_kernel in front of the lane <-> P kernels (g(1), g(s), g(m) read from
+    its rows instead of interpolated in every CTA), with a last group of message sizes that is not full, in both
+    segment-count modes; three tables are compared with the oracle."""
+    from dataclasses import replace
+    base = wl.config4(n_tables=320, P_hi=300, n_m=34, n_s=20, seed_offset=11)
+    for k_mode in (0, 1):
+        w = replace(base, k_mode=k_mode)
+        ot = oracle_tables(w)
+        import torch
+        with plogp.Tables.from_workload(w) as tabs:
+            dec = plogp.select_best(tabs, w)
+            pred = plogp.predict(tabs, w)
+            torch.cuda.synchronize()
+            n = check_decision(w, ot, dec, tables=[0, 157, 319]) + check_prediction(w, ot, pred, tables=[0, 157, 319])
+        assert n > 0
+
+
 def test_sweep_kernel_with_several_tables(plogp):
     """Long candidate list (512 multiples of 4 B) on three independent tables: the sweep kernel's table
     dimension and the reduction of its partial minima per table."""
