@@ -162,11 +162,11 @@ struct SegminParams {
     double *p_time;      // [n_tables][13][n_P][n_m]: planes 2, 5, 9 are written
     uint32_t *p_best_s;  // [n_tables][3][n_P][n_m], or nullptr
 };
-constexpr int kSegThreads = 128;
+constexpr int kSegThreads = 256;
 constexpr int kSegWarps = kSegThreads / 32;
 constexpr int kSegR = 8;                 // process counts per thread
 constexpr int kSegTileP = 32 * kSegR;    // process counts per CTA
-constexpr int kSegMG = 8;                // message sizes per CTA, two per warp
+constexpr int kSegMG = 16;               // message sizes per CTA, two per warp
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;

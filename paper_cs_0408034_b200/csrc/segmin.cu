@@ -3,20 +3,21 @@
 // of the model over the candidate segment sizes and the smallest size that attains it.
 //
 // Same building blocks as decide_kernel (decide.cu), with one running minimum per strategy instead of one
-// over all of them.  One CTA owns one table, 8 consecutive message sizes (two per warp) and a tile of 256
-// process counts (lane + 32 r, r = 0..7).  For a fixed message size the models are lines,
+// over all of them.  One CTA (8 warps) owns one table, 16 consecutive message sizes (two per warp) and a tile
+// of 256 process counts (lane + 32 r, r = 0..7).  For a fixed message size the models are lines,
 //     id 2: fma(P-1, Q, L)      id 9: fma(floor(log2 P), Q, ceil(log2 P) L)      Q = g(s) k
 //     id 5: fma(P-1, B, C)      B = g(s) + L, C = g(s) (k-1)
-// so a warp builds the coefficients of its message size once (lanes <-> candidates) and then sweeps each
-// strategy's list: every cell is evaluated with one DFMA and compared with the running minimum on the high
+// so a warp first builds the coefficient lists of its message sizes (lanes <-> candidates); then the CTA takes
+// one strategy at a time: every warp sweeps that strategy's list for its message sizes, the results are staged
+// in shared memory as [m][P], and the whole CTA writes the strategy's plane out as rows of 16 consecutive m
+// (128-byte row segments) before the next strategy reuses the staging area.  In a sweep
+// every cell is evaluated with one DFMA and compared with the running minimum on the high
 // 32 bits only, in the integer pipe (times are non-negative); a group of four candidates in which some cell
 // can reach the minimum is re-evaluated with the exact comparison, (time, candidate) in lexicographic order,
 // for the rows of 32 process counts that need it.  The running minima start from a pilot: for ids 2 and 9 the
 // candidate with the smallest Q, which is their winner for every P (the sweep still visits every cell), for
-// id 5 the winner at the tile's middle process count.
-//
-// Results are staged in shared memory as [strategy][m][P] and written out as rows of 8 consecutive m into
-// the prediction planes (time[table][13][P][m], best_s[table][3][P][m]).
+// id 5 the winner at the tile's middle process count.  The outputs are the prediction planes
+// time[table][13][P][m] and best_s[table][3][P][m].
 #include "device_common.cuh"
 
 #include <algorithm>
@@ -35,10 +36,11 @@ constexpr uint32_t kWhole = 0xFFFEu;     // no candidate fits: the whole message
 static_assert(kMaxInlineS <= 64, "warp_argmin_pilot keeps a candidate index in six bits");
 
 struct SegSmem {
-    double *tab, *gs, *gm, *lf, *lc, *pm1, *lq, *st_time;
-    double2 *l5;
+    double *tab, *gs, *gm, *lf, *lc, *pm1, *lq, *qp, *st_time;
+    double2 *l5, *ep;
     uint32_t *sval;
     uint16_t *st_idx;
+    int *pc;
     int cap;
 };
 
@@ -50,14 +52,17 @@ __host__ __device__ inline size_t seg_layout(int npad, int n_s, unsigned char *b
     auto take = [&](size_t bytes) { size_t at = off; off += (bytes + 15) & ~size_t(15); return at; };
     const size_t o_tab = take(3 * size_t(npad) * 8), o_gs = take(size_t(nsv) * 8), o_sv = take(size_t(nsv) * 4),
                  o_gm = take(kSegMG * 8), o_lf = take(kSegTileP * 8), o_lc = take(kSegTileP * 8), o_pm = take(kSegTileP * 8),
-                 o_lq = take(size_t(kSegWarps) * cap * 8), o_l5 = take(size_t(kSegWarps) * cap * 16),
-                 o_t = take(size_t(3) * kSegMG * kStride * 8), o_i = take(size_t(3) * kSegMG * kIStride * 2);
+                 o_lq = take(size_t(kSegMG) * cap * 8), o_l5 = take(size_t(kSegMG) * cap * 16),
+                 o_qp = take(kSegMG * 8), o_ep = take(kSegMG * 16), o_pc = take(2 * kSegMG * 4),
+                 o_t = take(size_t(kSegMG) * kStride * 8), o_i = take(size_t(kSegMG) * kIStride * 2);
     if (o) {
         o->tab = reinterpret_cast<double *>(base + o_tab); o->gs = reinterpret_cast<double *>(base + o_gs);
         o->sval = reinterpret_cast<uint32_t *>(base + o_sv); o->gm = reinterpret_cast<double *>(base + o_gm);
         o->lf = reinterpret_cast<double *>(base + o_lf); o->lc = reinterpret_cast<double *>(base + o_lc);
         o->pm1 = reinterpret_cast<double *>(base + o_pm);
         o->lq = reinterpret_cast<double *>(base + o_lq); o->l5 = reinterpret_cast<double2 *>(base + o_l5);
+        o->qp = reinterpret_cast<double *>(base + o_qp); o->ep = reinterpret_cast<double2 *>(base + o_ep);
+        o->pc = reinterpret_cast<int *>(base + o_pc);
         o->st_time = reinterpret_cast<double *>(base + o_t); o->st_idx = reinterpret_cast<uint16_t *>(base + o_i);
         o->cap = cap;
     }
@@ -85,14 +90,13 @@ __device__ __forceinline__ void offer(double &bt, uint32_t &bidx, double t, uint
 
 }  // namespace
 
-__global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminParams p)
+__global__ void __launch_bounds__(kSegThreads, 2) segmin_kernel(const SegminParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int npad = p.T.npad;
     SegSmem sm;
     seg_layout(npad, p.G.n_s, smem_raw, &sm);
     const uint32_t mask = p.G.mask;
-    const bool has2 = (mask >> 2) & 1u, has5 = (mask >> 5) & 1u, has9 = (mask >> 9) & 1u;
 
     int b = blockIdx.x;
     const int mgroup = b % p.n_mgroups;
@@ -129,9 +133,8 @@ __global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminPara
     __syncthreads();
 
     const double x_mid = sm.pm1[n_valid / 2];
-    double *lq = sm.lq + warp * sm.cap;
-    double2 *l5 = sm.l5 + warp * sm.cap;
 
+    // ---- phase 0: the coefficient lists of the warp's message sizes (lanes <-> candidates) and the pilots ----
     for (int mi = warp; mi < n_mi; mi += kSegWarps) {
         const int midx = m0 + mi;
         const int ns = p.G.ns_of_m[midx];
@@ -139,9 +142,8 @@ __global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminPara
         const int np = (nsv + U - 1) / U * U;
         const double gm = sm.gm[mi];
         const double *krow = p.G.k_list + static_cast<size_t>(midx) * p.G.n_s;
-
-        // ---- coefficients of this message size (lanes <-> candidates) and the pilots ----
-        __syncwarp();  // the previous message size's loops have finished reading the lists
+        double *lq = sm.lq + mi * sm.cap;
+        double2 *l5 = sm.l5 + mi * sm.cap;
         double qb = CUDART_INF, tb = CUDART_INF;
         int qc = kIntMax, tc = kIntMax;
         for (int c = lane; c < np; c += 32) {
@@ -172,124 +174,136 @@ __global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminPara
         if (lane == 0) {
             lq[qc] = CUDART_INF;
             l5[tc] = make_double2(CUDART_INF, CUDART_INF);
+            sm.qp[mi] = q_pilot; sm.ep[mi] = e_pilot;
+            sm.pc[2 * mi] = qc; sm.pc[2 * mi + 1] = tc;
         }
-        __syncwarp();
-        const uint32_t whole = ns > 0 ? 0u : 1u;
+    }
+    __syncwarp();  // the lists and pilots of a message size are read by the warp that wrote them
 
-        auto stage = [&](int q, const double *bt, const uint32_t *bidx) {
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                sm.st_time[(q * kSegMG + mi) * kStride + 32 * r + lane] = bt[r];
-                sm.st_idx[(q * kSegMG + mi) * kIStride + 32 * r + lane] = static_cast<uint16_t>(whole ? kWhole : bidx[r]);
-            }
-        };
-
-        // Filter of a group of U candidates: the smallest high word of the U times minus the high word of the running
-        // minimum says whether a cell can reach it (<= 0); the differences of all R process counts are folded into one
-        // integer minimum and one vote decides whether the group needs the exact pass.
-
-        // ---- ids 2 and 9: the list of Q, swept once per strategy ----
-        auto sweep_q = [&](auto is9_tag) {
-            constexpr bool IS9 = decltype(is9_tag)::value;
-            // id 2: fma(P-1, Q, L); id 9: fma(floor(log2 P), Q, ceil(log2 P) L)
-            double x[R], c9[IS9 ? R : 1];
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                x[r] = IS9 ? sm.lf[32 * r + lane] : sm.pm1[32 * r + lane];
-                if (IS9) c9[r] = sm.lc[32 * r + lane] * L;
-            }
-            if (!IS9) c9[0] = L;
-            double bt[R];
-            uint32_t bidx[R];
-#pragma unroll
-            for (int r = 0; r < R; ++r) { bt[r] = fma(x[r], q_pilot, c9[IS9 ? r : 0]); bidx[r] = static_cast<uint32_t>(qc); }
+    const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
+    const int ids[3] = {2, 5, 9};
+    // ---- one strategy at a time: every warp sweeps it for its message sizes, then the CTA writes the plane ----
 #pragma unroll 1
-            for (int j = 0; j < np; j += U) {
-                const double2 q01 = *reinterpret_cast<const double2 *>(lq + j), q23 = *reinterpret_cast<const double2 *>(lq + j + 2);
-                int acc = kIntMax;
+    for (int q = 0; q < 3; ++q) {
+        if (!((mask >> ids[q]) & 1u)) continue;
+        for (int mi = warp; mi < n_mi; mi += kSegWarps) {
+            const int midx = m0 + mi;
+            const int ns = p.G.ns_of_m[midx];
+            const int np = (max(ns, 1) + U - 1) / U * U;
+            const double *lq = sm.lq + mi * sm.cap;
+            const double2 *l5 = sm.l5 + mi * sm.cap;
+            const uint32_t whole = ns > 0 ? 0u : 1u;
+            auto stage = [&](const double *bt, const uint32_t *bidx) {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    const double c = c9[IS9 ? r : 0];
-                    const int h0 = hi32(fma(x[r], q01.x, c)), h1 = hi32(fma(x[r], q01.y, c));
-                    const int h2 = hi32(fma(x[r], q23.x, c)), h3 = hi32(fma(x[r], q23.y, c));
-                    acc = min(acc, min(min(h0, h1), min(h2, h3)) - hi32(bt[r]));
+                    sm.st_time[mi * kStride + 32 * r + lane] = bt[r];
+                    sm.st_idx[mi * kIStride + 32 * r + lane] = static_cast<uint16_t>(whole ? kWhole : bidx[r]);
                 }
-                if (__any_sync(kFull, acc <= 0)) {
+            };
+            // Filter of a group of U candidates: the smallest high word of the U times minus the high word of the running
+            // minimum says whether a cell can reach it (<= 0); the differences of all R process counts are folded into one
+            // integer minimum and one vote decides whether the group needs the exact pass.
+            auto sweep_q = [&](auto is9_tag) {
+                constexpr bool IS9 = decltype(is9_tag)::value;
+                // id 2: fma(P-1, Q, L); id 9: fma(floor(log2 P), Q, ceil(log2 P) L)
+                const double q_pilot = sm.qp[mi];
+                const int qc = sm.pc[2 * mi];
+                double x[R], c9[IS9 ? R : 1];
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    x[r] = IS9 ? sm.lf[32 * r + lane] : sm.pm1[32 * r + lane];
+                    if (IS9) c9[r] = sm.lc[32 * r + lane] * L;
+                }
+                if (!IS9) c9[0] = L;
+                double bt[R];
+                uint32_t bidx[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) { bt[r] = fma(x[r], q_pilot, c9[IS9 ? r : 0]); bidx[r] = static_cast<uint32_t>(qc); }
+#pragma unroll 1
+                for (int j = 0; j < np; j += U) {
+                    const double2 q01 = *reinterpret_cast<const double2 *>(lq + j), q23 = *reinterpret_cast<const double2 *>(lq + j + 2);
+                    int acc = kIntMax;
 #pragma unroll
                     for (int r = 0; r < R; ++r) {
                         const double c = c9[IS9 ? r : 0];
                         const int h0 = hi32(fma(x[r], q01.x, c)), h1 = hi32(fma(x[r], q01.y, c));
                         const int h2 = hi32(fma(x[r], q23.x, c)), h3 = hi32(fma(x[r], q23.y, c));
-                        if (__any_sync(kFull, min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]))) {
-#pragma unroll 1
-                            for (int u = 0; u < U; ++u) offer(bt[r], bidx[r], fma(x[r], lq[j + u], c), static_cast<uint32_t>(j + u));
-                        }
+                        acc = min(acc, min(min(h0, h1), min(h2, h3)) - hi32(bt[r]));
                     }
-                }
-            }
-            stage(IS9 ? 2 : 0, bt, bidx);
-        };
-        if (has2) sweep_q(std::false_type{});
-        if (has9) sweep_q(std::true_type{});
-
-        // ---- id 5: list of (B, C) ----
-        if (has5) {
-            double pm1[R], bt[R];
-            uint32_t bidx[R];
+                    if (__any_sync(kFull, acc <= 0)) {
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                pm1[r] = sm.pm1[32 * r + lane];
-                bt[r] = fma(pm1[r], e_pilot.x, e_pilot.y);
-                bidx[r] = static_cast<uint32_t>(tc);
-            }
+                        for (int r = 0; r < R; ++r) {
+                            const double c = c9[IS9 ? r : 0];
+                            const int h0 = hi32(fma(x[r], q01.x, c)), h1 = hi32(fma(x[r], q01.y, c));
+                            const int h2 = hi32(fma(x[r], q23.x, c)), h3 = hi32(fma(x[r], q23.y, c));
+                            if (__any_sync(kFull, min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]))) {
 #pragma unroll 1
-            for (int j = 0; j < np; j += U) {
-                const double2 e0 = l5[j], e1 = l5[j + 1], e2 = l5[j + 2], e3 = l5[j + 3];
-                int acc = kIntMax;
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const int h0 = hi32(fma(pm1[r], e0.x, e0.y)), h1 = hi32(fma(pm1[r], e1.x, e1.y));
-                    const int h2 = hi32(fma(pm1[r], e2.x, e2.y)), h3 = hi32(fma(pm1[r], e3.x, e3.y));
-                    acc = min(acc, min(min(h0, h1), min(h2, h3)) - hi32(bt[r]));
-                }
-                if (__any_sync(kFull, acc <= 0)) {
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        const int h0 = hi32(fma(pm1[r], e0.x, e0.y)), h1 = hi32(fma(pm1[r], e1.x, e1.y));
-                        const int h2 = hi32(fma(pm1[r], e2.x, e2.y)), h3 = hi32(fma(pm1[r], e3.x, e3.y));
-                        if (__any_sync(kFull, min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]))) {
-#pragma unroll 1
-                            for (int u = 0; u < U; ++u) {
-                                const double2 e = l5[j + u];
-                                offer(bt[r], bidx[r], fma(pm1[r], e.x, e.y), static_cast<uint32_t>(j + u));
+                                for (int u = 0; u < U; ++u) offer(bt[r], bidx[r], fma(x[r], lq[j + u], c), static_cast<uint32_t>(j + u));
                             }
                         }
                     }
                 }
-            }
-            stage(1, bt, bidx);
-        }
-    }
-    __syncthreads();
-
-    // transposed write-out: rows of 8 consecutive m per process count and strategy
-    const size_t plane = static_cast<size_t>(p.G.n_P) * p.G.n_m;
-    const int ids[3] = {2, 5, 9};
-    if (p.vec_out) {
-        // two message sizes per lane (16-byte and 8-byte stores; the host has checked the alignment), running pointers
-        constexpr int kHalf = kSegMG / 2, kRows = 32 / kHalf, kStep = kSegWarps * kRows;
-        const int mi = 2 * (lane & (kHalf - 1)), pr0 = warp * kRows + lane / kHalf;
-        if (mi < n_mi) {  // n_m is even, so mi + 1 is a message size of the grid too
-            const uint32_t m_u0 = p.G.m_list[m0 + mi], m_u1 = p.G.m_list[m0 + mi + 1];
-            const size_t cell0 = static_cast<size_t>(tile0 + pr0) * p.G.n_m + static_cast<size_t>(m0 + mi);
-            const size_t step = static_cast<size_t>(kStep) * p.G.n_m;
+                stage(bt, bidx);
+            };
+            if (q == 0) sweep_q(std::false_type{});
+            else if (q == 2) sweep_q(std::true_type{});
+            else {
+                // ---- id 5: list of (B, C) ----
+                const double2 e_pilot = sm.ep[mi];
+                const int tc = sm.pc[2 * mi + 1];
+                double pm1[R], bt[R];
+                uint32_t bidx[R];
 #pragma unroll
-            for (int q = 0; q < 3; ++q) {
-                if (!((mask >> ids[q]) & 1u)) continue;
-                const double *st0 = sm.st_time + (q * kSegMG + mi) * kStride + pr0, *st1 = st0 + kStride;
-                const uint16_t *si0 = sm.st_idx + (q * kSegMG + mi) * kIStride + pr0, *si1 = si0 + kIStride;
-                double *out_t = p.p_time + (static_cast<size_t>(table - p.out_table0) * 13 + ids[q]) * plane + cell0;
-                uint32_t *out_s = p.p_best_s ? p.p_best_s + (static_cast<size_t>(table - p.out_table0) * 3 + q) * plane + cell0 : nullptr;
+                for (int r = 0; r < R; ++r) {
+                    pm1[r] = sm.pm1[32 * r + lane];
+                    bt[r] = fma(pm1[r], e_pilot.x, e_pilot.y);
+                    bidx[r] = static_cast<uint32_t>(tc);
+                }
+#pragma unroll 1
+                for (int j = 0; j < np; j += U) {
+                    const double2 e0 = l5[j], e1 = l5[j + 1], e2 = l5[j + 2], e3 = l5[j + 3];
+                    int acc = kIntMax;
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const int h0 = hi32(fma(pm1[r], e0.x, e0.y)), h1 = hi32(fma(pm1[r], e1.x, e1.y));
+                        const int h2 = hi32(fma(pm1[r], e2.x, e2.y)), h3 = hi32(fma(pm1[r], e3.x, e3.y));
+                        acc = min(acc, min(min(h0, h1), min(h2, h3)) - hi32(bt[r]));
+                    }
+                    if (__any_sync(kFull, acc <= 0)) {
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            const int h0 = hi32(fma(pm1[r], e0.x, e0.y)), h1 = hi32(fma(pm1[r], e1.x, e1.y));
+                            const int h2 = hi32(fma(pm1[r], e2.x, e2.y)), h3 = hi32(fma(pm1[r], e3.x, e3.y));
+                            if (__any_sync(kFull, min(min(h0, h1), min(h2, h3)) <= hi32(bt[r]))) {
+#pragma unroll 1
+                                for (int u = 0; u < U; ++u) {
+                                    const double2 e = l5[j + u];
+                                    offer(bt[r], bidx[r], fma(pm1[r], e.x, e.y), static_cast<uint32_t>(j + u));
+                                }
+                            }
+                        }
+                    }
+                }
+                stage(bt, bidx);
+            }
+        }
+        __syncthreads();
+
+        // transposed write-out of the strategy's plane: rows of 16 consecutive m per process count
+        double *plane_t = p.p_time + (static_cast<size_t>(table - p.out_table0) * 13 + ids[q]) * plane;
+        uint32_t *plane_s = p.p_best_s ? p.p_best_s + (static_cast<size_t>(table - p.out_table0) * 3 + q) * plane : nullptr;
+        if (p.vec_out) {
+            // two message sizes per lane (16-byte and 8-byte stores; the host has checked the alignment), running pointers
+            constexpr int kHalf = kSegMG / 2, kRows = 32 / kHalf, kStep = kSegWarps * kRows;
+            const int mi = 2 * (lane & (kHalf - 1)), pr0 = warp * kRows + lane / kHalf;
+            if (mi < n_mi) {  // n_m is even, so mi + 1 is a message size of the grid too
+                const uint32_t m_u0 = p.G.m_list[m0 + mi], m_u1 = p.G.m_list[m0 + mi + 1];
+                const size_t cell0 = static_cast<size_t>(tile0 + pr0) * p.G.n_m + static_cast<size_t>(m0 + mi);
+                const size_t step = static_cast<size_t>(kStep) * p.G.n_m;
+                const double *st0 = sm.st_time + mi * kStride + pr0, *st1 = st0 + kStride;
+                const uint16_t *si0 = sm.st_idx + mi * kIStride + pr0, *si1 = si0 + kIStride;
+                double *out_t = plane_t + cell0;
+                uint32_t *out_s = plane_s ? plane_s + cell0 : nullptr;
                 for (int pr = pr0; pr < n_valid; pr += kStep) {
                     *reinterpret_cast<double2 *>(out_t) = make_double2(*st0, *st1);
                     if (out_s) {
@@ -301,29 +315,23 @@ __global__ void __launch_bounds__(kSegThreads, 3) segmin_kernel(const SegminPara
                     st0 += kStep; st1 += kStep; si0 += kStep; si1 += kStep;
                 }
             }
-        }
-    } else {
-        const int mi = lane & (kSegMG - 1), prow = lane / kSegMG, rows = 32 / kSegMG;
-        if (mi < n_mi) {
-            const uint32_t m_u = p.G.m_list[m0 + mi];
-            const size_t cell0 = static_cast<size_t>(m0 + mi);
-#pragma unroll
-            for (int q = 0; q < 3; ++q) {
-                if (!((mask >> ids[q]) & 1u)) continue;
-                const double *st = sm.st_time + (q * kSegMG + mi) * kStride;
-                const uint16_t *si = sm.st_idx + (q * kSegMG + mi) * kIStride;
-                double *out_t = p.p_time + (static_cast<size_t>(table - p.out_table0) * 13 + ids[q]) * plane + cell0;
-                uint32_t *out_s = p.p_best_s ? p.p_best_s + (static_cast<size_t>(table - p.out_table0) * 3 + q) * plane + cell0 : nullptr;
+        } else {
+            const int mi = lane & (kSegMG - 1), prow = lane / kSegMG, rows = 32 / kSegMG;
+            if (mi < n_mi) {
+                const uint32_t m_u = p.G.m_list[m0 + mi];
+                const double *st = sm.st_time + mi * kStride;
+                const uint16_t *si = sm.st_idx + mi * kIStride;
                 for (int pr = warp * rows + prow; pr < n_valid; pr += kSegWarps * rows) {
-                    const size_t o = static_cast<size_t>(tile0 + pr) * p.G.n_m;
-                    out_t[o] = st[pr];
-                    if (out_s) {
+                    const size_t o = static_cast<size_t>(tile0 + pr) * p.G.n_m + static_cast<size_t>(m0 + mi);
+                    plane_t[o] = st[pr];
+                    if (plane_s) {
                         const uint32_t idx = si[pr];
-                        out_s[o] = idx == kWhole ? m_u : sm.sval[idx];
+                        plane_s[o] = idx == kWhole ? m_u : sm.sval[idx];
                     }
                 }
             }
         }
+        __syncthreads();  // the staging area is free again
     }
 }
 
