@@ -38,7 +38,7 @@ NOMINAL_FP64_FMA_RATE = 148 * 64 * 1.965e9  # SMs x FP64 lanes per SM x max SM c
 # under profiles/ (batched workload cut to 1024 tables: 0.87 GB of output per kernel, far beyond the L2,
 # so what is still cached when the kernel ends is a few percent; traffic grows in proportion to the table
 # count).  An entry is None while its kernel has changed since the last capture.
-NCU_TRAFFIC_BYTES_PER_TABLE = {"decide_kernel": (814.151424e6 + 1.608960e6) / 1024, "scatter_kernel": (812.180992e6 + 1.666560e6) / 1024,
+NCU_TRAFFIC_BYTES_PER_TABLE = {"decide_kernel": (813.820672e6 + 1.456128e6) / 1024, "scatter_kernel": (812.184320e6 + 1.679872e6) / 1024,
                                "sweep_kernel": None}
 NCU_TRAFFIC_NOTE = "bytes per launch = bytes per table of the 1024-table ncu capture in profiles/ x tables"
 FALLBACK_HBM_GBS = 6650.0
