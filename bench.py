@@ -401,6 +401,43 @@ class Bench:
                              "frac": nbytes / (self.hbm_gbs * 1e9) / (ms * 1e-3), "algorithmic_bytes": nbytes,
                              "peak_source": "HBM copy bandwidth, of %s" % self.peak_src}}
 
+    def graph_entries(self):
+        """The launch-bound grids again, replayed from a captured CUDA graph: with its plan cached a call only
+        launches kernels on the caller's stream, so a loop of calls can be captured once and replayed.  Back-to-back
+        calls (no L2 flush between them), device time per call, next to the same loop of direct calls."""
+        plogp, torch = self.plogp, self.torch
+        out = []
+        for w in (wl.config1(), wl.config2(), wl.config5()):
+            with plogp.Tables.from_workload(w) as tabs:
+                g = plogp.GridArgs.from_workload(w)
+                dec = plogp.select_best(tabs, g)  # builds the plan, allocates scratch
+                torch.cuda.synchronize()
+                st = torch.cuda.Stream()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(st):
+                    plogp.select_best(tabs, g, out=dec, stream=st)
+                    st.synchronize()
+                    with torch.cuda.graph(graph, stream=st):
+                        plogp.select_best(tabs, g, out=dec, stream=st)
+                n = 200
+
+                def per_call(fn):
+                    for _ in range(10):
+                        fn()
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    for _ in range(n):
+                        fn()
+                    b.record()
+                    b.synchronize()
+                    return a.elapsed_time(b) / n
+                t_graph = per_call(graph.replay)
+                t_direct = per_call(lambda: plogp.select_best(tabs, g, out=dec))
+                out.append({"workload": w.name, "calls": n, "ms_per_call_graph_replay": t_graph, "ms_per_call_direct": t_direct,
+                            "note": "back-to-back calls, no L2 flush"})
+                del graph
+        return out
+
     def aux_entries(self, w4):
         """The segment-size sensitivity calls: the model surface over s on the dense single-table grid, the fixed
         8 kB segment size and the decision boundaries on the batched workload."""
@@ -592,6 +629,7 @@ def run_ours(args, rank, local_rank, world):
                                            "skipped cells are not counted as model cells"))
         line["workloads"] = others
         line["sensitivity_calls"] = b.aux_entries(w)
+        line["graph_replay"] = b.graph_entries()
     if world == 1 and not args.no_cpu_baseline:
         v, cores, text = oracle_sample_rate(w, 15.0)
         v1, _, text1 = oracle_sample_rate(w, 8.0, threads=1)

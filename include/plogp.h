@@ -132,6 +132,10 @@ typedef struct {
  *   stream    a cudaStream_t (NULL = default stream).  Work is enqueued; the call does not wait
  *             for it, but may synchronise when the handle's scratch has to grow.
  * Both outputs belong to the caller.
+ * The handle keeps the launch plan of the last grid: a call with the same grid (and per-kernel
+ * timing off) copies nothing and allocates nothing, it only launches kernels on `stream`, so a
+ * loop of such calls may be captured into a CUDA graph and replayed.  The first call with a new
+ * grid uploads the grid and may allocate scratch: make it outside the capture.
  */
 int plogp_predict(plogp_tables *tables, const plogp_grid *grid, double *d_time, uint32_t *d_best_s,
                   void *stream);

@@ -233,6 +233,36 @@ def test_many_tables_take_the_gap_prepass(plogp):
         assert n > 0
 
 
+def test_repeated_call_can_be_replayed_from_a_cuda_graph(plogp):
+    """With its plan cached a call only launches kernels on the caller's stream, so it can be captured into a CUDA
+    graph and replayed; the replay must reproduce the direct call bit for bit (decision kernel and Scatter kernels)."""
+    import torch
+    for w in (wl.config1(), wl.config5(P_hi=3000, n_m=40)):
+        with plogp.Tables.from_workload(w) as tabs:
+            dec = plogp.select_best(tabs, w)  # builds the plan, allocates scratch
+            torch.cuda.synchronize()
+            st = torch.cuda.Stream()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(st):
+                plogp.select_best(tabs, w, out=dec, stream=st)
+                st.synchronize()
+                with torch.cuda.graph(graph, stream=st):
+                    plogp.select_best(tabs, w, out=dec, stream=st)
+            for t in (dec.strategy, dec.s_bytes, dec.time):
+                t.zero_()
+            plogp.select_best(tabs, w, out=dec)
+            torch.cuda.synchronize()
+            ref = (dec.strategy.clone(), dec.s_bytes.clone(), dec.time.clone())
+            for t in (dec.strategy, dec.s_bytes, dec.time):
+                t.zero_()
+            torch.cuda.synchronize()
+            graph.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(dec.strategy, ref[0]) and torch.equal(dec.s_bytes, ref[1])
+            assert torch.equal(dec.time.view(torch.int64), ref[2].view(torch.int64))
+            del graph
+
+
 def test_sweep_kernel_with_several_tables(plogp):
     """Long candidate list (512 multiples of 4 B) on three independent tables: the sweep kernel's table
     dimension and the reduction of its partial minima per table."""
