@@ -263,6 +263,37 @@ def test_repeated_call_can_be_replayed_from_a_cuda_graph(plogp):
             del graph
 
 
+def test_randomised_grids_against_the_oracle(plogp):
+    """Forty seeded random grids (1-5 tables; ranges, sub-ranges and lists of process counts that end inside, at and
+    past a tile of 256; 1-40 message sizes; 1-64 candidates, some grids with message sizes below every candidate;
+    random strategy masks; both segment-count modes and both search modes): decision table and predictions of every
+    cell against the oracle."""
+    from dataclasses import replace
+    import torch
+    rng = np.random.default_rng(408034)
+    for case in range(40):
+        nt = int(rng.integers(1, 6))
+        P_hi = int(rng.choice([3, 9, 33, 70, 257, 300, 513, 600]))
+        base = wl.config4(n_tables=nt, P_hi=P_hi, n_m=int(rng.integers(1, 41)), n_s=int(rng.integers(1, 65)), seed_offset=1000 + case)
+        mask = wl.ALL_STRATEGIES if rng.random() < 0.3 else int(rng.integers(1, 1 << 13))
+        kw = dict(strategy_mask=mask, k_mode=int(rng.integers(0, 2)), search_mode=int(rng.integers(0, 2)))
+        pick = rng.random()
+        if pick < 0.3:
+            Ps = np.unique(rng.integers(2, P_hi + 1, size=int(rng.integers(1, 30)))).astype(np.int32)
+            kw.update(P_list=Ps, P_lo=int(Ps[0]), P_hi=int(Ps[-1]))
+        elif pick < 0.6:
+            kw.update(P_lo=int(rng.integers(2, P_hi + 1)))
+        if rng.random() < 0.2:
+            kw.update(s_list=wl.log_spaced_multiples(1 << 10, 1 << 20, len(base.s_list)))
+        w = replace(base, **kw)
+        ot = oracle_tables(w)
+        with plogp.Tables.from_workload(w) as tabs:
+            dec = plogp.select_best(tabs, w)
+            pred = plogp.predict(tabs, w)
+            torch.cuda.synchronize()
+            assert check_decision(w, ot, dec) + check_prediction(w, ot, pred) > 0, case
+
+
 def test_sweep_kernel_with_several_tables(plogp):
     """Long candidate list (512 multiples of 4 B) on three independent tables: the sweep kernel's table
     dimension and the reduction of its partial minima per table."""
